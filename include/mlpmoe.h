@@ -1,0 +1,228 @@
+/*
+ * mlpmoe.h - C ABI of the B200 (sm_100a) MLPMoE forward library.
+ *
+ * The layer (arXiv 2511.21089, Section 3.1):
+ *     MLPMoE(x) = sum_b alpha_b * W_down^(b) [ silu(W_gate^(b) x) (.) W_up^(b) x ]
+ * over B contiguous slices of the intermediate dimension, with Fractal Fade
+ * (Section 3.2) and Compensated Branch Pruning (Section 3.3) applied to the
+ * weights / gates before the forward pass.
+ *
+ * Conventions for every call
+ *   - "device" pointers are CUDA device memory of the current device, owned by the
+ *     caller unless stated otherwise; "host" pointers are ordinary host memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - Every call returns a status; nothing throws or aborts across this boundary.
+ *     On error no state of the handle changes.
+ *   - One handle may be used from one stream at a time.
+ *   - There is no CPU fallback: without a usable CUDA device every compute call
+ *     returns MLPMOE_ERR_CUDA.
+ *   - Inputs are assumed finite (skipping zeroed work is exact only then).
+ */
+#ifndef MLPMOE_H_
+#define MLPMOE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mlpmoe_layer_s* mlpmoe_handle_t;
+
+typedef enum {
+  MLPMOE_OK = 0,
+  MLPMOE_ERR_INVALID_ARG = 1,     /* NULL pointer, negative size, n_tokens > max_tokens, misaligned buffer */
+  MLPMOE_ERR_BAD_PARTITION = 2,   /* sum d_b != d_inter, d_b <= 0, or d_b not a multiple of 16 */
+  MLPMOE_ERR_EMPTY_KEEP_SET = 3,  /* pruning would leave no branch */
+  MLPMOE_ERR_BAD_SCHEDULE = 4,    /* a sparsity ratio outside [0, 1) */
+  MLPMOE_ERR_UNSUPPORTED = 5,     /* shape or dtype combination the kernels do not cover */
+  MLPMOE_ERR_ALLOC = 6,           /* device or host allocation failed */
+  MLPMOE_ERR_CUDA = 7,            /* a CUDA runtime / driver call failed (includes: no device) */
+  MLPMOE_ERR_DEVICE_TIMEOUT = 8   /* a bounded wait inside a kernel ran out (see mlpmoe_get_status) */
+} mlpmoe_status_t;
+
+typedef enum { MLPMOE_BF16 = 0, MLPMOE_FP32 = 1 } mlpmoe_dtype_t;
+
+typedef enum {
+  MLPMOE_LAYOUT_PAPER = 0,  /* W_gate, W_up: [d_model x d_inter]; W_down: [d_inter x d_model]; row-major (Section 3.1) */
+  MLPMOE_LAYOUT_LINEAR = 1  /* [out x in] row-major: gate/up [d_inter x d_model], down [d_model x d_inter] */
+} mlpmoe_layout_t;
+
+/* ------------------------------------------------------------------------- *
+ * Set-up calls (may synchronise the stream; allocate library-owned memory)
+ * ------------------------------------------------------------------------- */
+
+/*
+ * Build a layer from dense SwiGLU weights (Section 3.1: partition of d_inter into
+ * B contiguous slices d_inter = sum_b d_b, sub-matrices by slicing, one scalar
+ * gate alpha_b per branch).
+ *   out        host: receives the handle (NULL on error).
+ *   d_b        host, length B: slice widths; each must be a positive multiple of 16.
+ *   W_gate, W_up, W_down   device, `dtype` elements in `layout`; copied and packed
+ *              on `stream`; the caller may free them once that stream work is done.
+ *   alpha      host, length B, or NULL for all 1.0 (the paper's initial value).
+ *   dtype      MLPMOE_BF16: bf16 weights and activations, fp32 accumulation on the
+ *              tensor cores; MLPMOE_FP32: fp32 everywhere (plain FMA arithmetic).
+ *   max_tokens largest n_tokens a later forward call may pass (sizes the
+ *              library-owned intermediate-activation workspace).
+ * d_model must be a multiple of 8.
+ */
+mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_inter,
+                              int32_t B, const int64_t* d_b,
+                              const void* W_gate, const void* W_up, const void* W_down,
+                              const float* alpha, mlpmoe_dtype_t dtype, mlpmoe_layout_t layout,
+                              int64_t max_tokens, void* stream);
+
+/* Free everything the handle owns.  NULL is allowed. */
+void mlpmoe_destroy(mlpmoe_handle_t h);
+
+/*
+ * Let `h` use `donor`'s intermediate-activation workspace instead of its own (a
+ * stack of layers that run one after another on one stream needs only one).
+ * `donor` must have been created with at least h's d_inter and max_tokens and
+ * the same dtype, and must outlive `h`.  Not in the paper: memory management only.
+ */
+mlpmoe_status_t mlpmoe_share_workspace(mlpmoe_handle_t h, mlpmoe_handle_t donor);
+
+/*
+ * Fractal Fade (Section 3.2, and the "Differential Sparsity Logic" fragment of
+ * Section 4): for every branch b with s_b > 0, and separately for its W_gate and
+ * its W_up slice (m = d_model * d_b entries each), zero every entry whose
+ * magnitude is not above the slice's s_b-quantile of magnitudes.  The quantile
+ * position is p = s_b (m - 1) in exact arithmetic; with lo = floor(p) the entries
+ * zeroed are exactly those with |w| <= (lo-th smallest |w|), ties included, which
+ * is the same set the linearly interpolated threshold with a strict '>' gives.
+ * W_down is not touched.  Applied in place to the library's copy; idempotent.
+ *   s   host, length B, each in [0, 1); 0 = leave the branch untouched.
+ *       NULL = the paper's schedule s_b = 0.9 b / B (b = 0 is the dense backbone),
+ *       evaluated in integer arithmetic as lo = (9 b (m - 1)) div (10 B).
+ * Afterwards neurons whose gate column, up column or down row is entirely zero are
+ * dropped from the schedule.  Synchronises `stream`.
+ */
+mlpmoe_status_t mlpmoe_fade(mlpmoe_handle_t h, const double* s, void* stream);
+
+/*
+ * Compensated Branch Pruning (Section 3.3) with an arbitrary keep set:
+ * alpha_b <- alpha_b(create) * sqrt(B / K) for kept branches (K = number kept;
+ * factor 1 if `compensate` is 0) and 0 for the others, computed as
+ * (float)(sqrt((double)B / K) * (double)alpha_b).  Always starts from the alpha
+ * given at create, so repeated calls do not accumulate.  Dropped branches are
+ * removed from the packed operands: their work is skipped, not masked.
+ *   keep  host, length B, non-zero = keep.  An empty keep set is an error.
+ * Synchronises `stream`.
+ */
+mlpmoe_status_t mlpmoe_prune(mlpmoe_handle_t h, const uint8_t* keep, int32_t compensate, void* stream);
+
+/* The paper's literal rule (Section 3.3): keep branches b < K, alpha_b = sqrt(B/K). 1 <= K <= B. */
+mlpmoe_status_t mlpmoe_prune_first_k(mlpmoe_handle_t h, int32_t K, void* stream);
+
+/* ------------------------------------------------------------------------- *
+ * Forward (Section 3.1 layer equation).  Enqueues on `stream`, never
+ * synchronises, allocates nothing.
+ * ------------------------------------------------------------------------- */
+
+/*
+ *   x  device, [n_tokens x d_model] row-major, the layer's dtype, 16-byte aligned.
+ *   y  device, [n_tokens x d_model] row-major, fp32, 16-byte aligned.
+ * n_tokens = 0 is a no-op; n_tokens > max_tokens is MLPMOE_ERR_INVALID_ARG.
+ * bf16 layers use the tensor-core GEMM pair for n_tokens > 64 and the
+ * weight-streaming decode kernels for n_tokens <= 64.
+ */
+mlpmoe_status_t mlpmoe_forward(mlpmoe_handle_t h, const void* x, void* y, int64_t n_tokens, void* stream);
+
+/*
+ * As mlpmoe_forward, with
+ *   residual  device fp32 [n_tokens x d_model] or NULL: y = residual + MLPMoE(x)
+ *             (may alias y when y_dtype is fp32);
+ *   y_dtype   MLPMOE_FP32, or MLPMOE_BF16 for a bf16 layer.
+ */
+mlpmoe_status_t mlpmoe_forward_ex(mlpmoe_handle_t h, const void* x, void* y, int64_t n_tokens,
+                                  const float* residual, mlpmoe_dtype_t y_dtype, void* stream);
+
+/*
+ * mlpmoe_forward on HOST buffers: copies x to the device, runs the layer, copies y
+ * back and synchronises `stream`.  x_host: layer dtype, y_host: fp32.  Pinned host
+ * memory makes the copies asynchronous; pageable memory works too.
+ */
+mlpmoe_status_t mlpmoe_forward_host(mlpmoe_handle_t h, const void* x_host, float* y_host,
+                                    int64_t n_tokens, void* stream);
+
+/* ------------------------------------------------------------------------- *
+ * Stack harness (not in the paper; the benchmark configurations wrap the layer
+ * as x <- x + MLPMoE_l(RMSNorm(x)), unit gain)
+ * ------------------------------------------------------------------------- */
+
+/* r[t,:] = x[t,:] / sqrt(mean(x[t,:]^2) + eps); x device fp32 [n x d]; r device [n x d] of out_dtype. */
+mlpmoe_status_t mlpmoe_rmsnorm(const float* x, void* r, int64_t n_tokens, int64_t d_model, float eps,
+                               mlpmoe_dtype_t out_dtype, void* stream);
+
+/*
+ * Run n_layers layers (all with the same d_model and dtype) over the fp32 residual
+ * stream x [n_tokens x d_model], in place: for each layer, RMSNorm into a
+ * library-owned buffer of the layer dtype, then x = x + MLPMoE_l(that).
+ */
+mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_layers, float* x,
+                                     int64_t n_tokens, float eps, void* stream);
+
+/* mlpmoe_stack_forward on HOST buffers (fp32 in, fp32 out); synchronises `stream`. */
+mlpmoe_status_t mlpmoe_stack_forward_host(const mlpmoe_handle_t* layers, int32_t n_layers,
+                                          const float* x_host, float* y_host,
+                                          int64_t n_tokens, float eps, void* stream);
+
+/* ------------------------------------------------------------------------- *
+ * Queries (host outputs; used by the parity harness)
+ * ------------------------------------------------------------------------- */
+
+/*
+ * The schedule: surviving branches in ascending order and the maximal runs of
+ * live neurons inside them (start index in 0..d_inter-1, length); their
+ * concatenation is the contraction index space of the down projection.
+ * branches: capacity B; seg_start / seg_len: capacity d_inter.  Any output may be NULL.
+ */
+mlpmoe_status_t mlpmoe_get_klist(mlpmoe_handle_t h, int32_t* branches, int32_t* n_branches,
+                                 int64_t* seg_start, int64_t* seg_len, int32_t* n_segs);
+/* Effective alpha_b (after pruning / compensation), length B. */
+mlpmoe_status_t mlpmoe_get_alpha(mlpmoe_handle_t h, float* alpha);
+/* Number of surviving (scheduled) intermediate neurons. */
+mlpmoe_status_t mlpmoe_get_active_neurons(mlpmoe_handle_t h, int64_t* n_active);
+/* Non-zero entries per branch of each projection (length B each; any may be NULL). Synchronises. */
+mlpmoe_status_t mlpmoe_nnz(mlpmoe_handle_t h, int64_t* nnz_gate, int64_t* nnz_up, int64_t* nnz_down);
+/*
+ * Copy the library's current weights back in the paper's layout (W_gate, W_up:
+ * [d_model x d_inter], W_down: [d_inter x d_model], layer dtype, device buffers;
+ * any may be NULL).  After mlpmoe_fade these hold the masked weights.
+ */
+mlpmoe_status_t mlpmoe_get_weights(mlpmoe_handle_t h, void* W_gate, void* W_up, void* W_down, void* stream);
+/*
+ * Reads the handle's device status word (synchronises the device): MLPMOE_OK, or
+ * MLPMOE_ERR_DEVICE_TIMEOUT if a bounded wait in a kernel expired since create.
+ */
+mlpmoe_status_t mlpmoe_get_status(mlpmoe_handle_t h);
+/* Kernels launched on behalf of this handle since create (forward calls only). */
+mlpmoe_status_t mlpmoe_get_launch_count(mlpmoe_handle_t h, int64_t* launches);
+const char* mlpmoe_status_string(mlpmoe_status_t s);
+
+/* ------------------------------------------------------------------------- *
+ * Host-only helpers: the scheduler's integer logic without any CUDA call
+ * ------------------------------------------------------------------------- */
+
+/* lo = floor(s (m - 1)) in exact arithmetic on the double s (Section 3.2 quantile position). */
+mlpmoe_status_t mlpmoe_host_fade_position(double s, int64_t m, int64_t* lo);
+/* lo for the paper's schedule s_b = 0.9 b / B: (9 b (m - 1)) div (10 B). */
+mlpmoe_status_t mlpmoe_host_fade_position_default(int32_t b, int32_t B, int64_t m, int64_t* lo);
+/* Effective gates of Section 3.3 from create-time alpha and a keep mask. */
+mlpmoe_status_t mlpmoe_host_prune_alpha(int32_t B, const float* alpha, const uint8_t* keep,
+                                        int32_t compensate, float* alpha_eff);
+/*
+ * Build the schedule from effective gates and per-neuron liveness flags
+ * (live: host uint8[d_inter] or NULL = all live).  Outputs as mlpmoe_get_klist.
+ */
+mlpmoe_status_t mlpmoe_host_schedule(int32_t B, const int64_t* d_b, const float* alpha_eff,
+                                     const uint8_t* live, int32_t* branches, int32_t* n_branches,
+                                     int64_t* seg_start, int64_t* seg_len, int32_t* n_segs,
+                                     int64_t* n_active);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MLPMOE_H_ */

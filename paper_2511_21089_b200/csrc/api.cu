@@ -1,0 +1,643 @@
+// C-ABI entry points and the host side of the library: argument checks, the weight packer's
+// control flow, the branch scheduler (Section 3.3 -> K-list), Fade set-up (Section 3.2) and the
+// dispatch of mlpmoe_forward onto the prefill / decode / fp32 kernels.
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/mlpmoe.h"
+#include "internal.h"
+
+using namespace mlpmoe;
+
+namespace {
+
+#define CK(expr)                                   \
+  do {                                             \
+    cudaError_t e__ = (expr);                      \
+    if (e__ != cudaSuccess) return MLPMOE_ERR_CUDA; \
+  } while (0)
+
+inline int64_t round_up(int64_t a, int64_t b) { return (a + b - 1) / b * b; }
+
+// Activation workspace; may be shared by the layers of a stack.
+struct Workspace {
+  void* H = nullptr;       // [max_tokens x Ipad_max] layer dtype: silu(gate)*up*scale
+  void* xnorm = nullptr;   // [max_tokens x d] layer dtype: RMSNorm output / host-call staging of x
+  float* yres = nullptr;   // [max_tokens x d] fp32: host-call staging of y / the residual stream
+  int64_t max_tokens = 0, Ipad_max = 0, d = 0;
+  int elem_size = 0;
+  int refs = 0;
+};
+
+void ws_release(Workspace* w) {
+  if (!w) return;
+  if (--w->refs > 0) return;
+  cudaFree(w->H);
+  cudaFree(w->xnorm);
+  cudaFree(w->yres);
+  delete w;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(p);
+  return fn;
+}
+
+// bf16 row-major matrix [outer x inner] with row pitch `pitch_elems`; box = 64 x box_outer, 128-byte swizzle.
+bool make_tmap(CUtensorMap* m, const void* ptr, int64_t inner, int64_t outer, int64_t pitch_elems, int box_outer) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(inner), static_cast<cuuint64_t>(outer)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch_elems) * 2};
+  cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_outer)};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// ------------------------------------------------------------ host logic ----
+// floor(s * (m - 1)) on the exact value of the double s, 0 <= s < 1.
+int64_t fade_position_exact(double s, int64_t m) {
+  if (s <= 0.0 || m <= 1) return 0;
+  int exp = 0;
+  const double mant = std::frexp(s, &exp);                       // s = mant * 2^exp, mant in [0.5, 1)
+  const unsigned long long M = static_cast<unsigned long long>(std::ldexp(mant, 53));   // exact: 53-bit integer
+  const int shift = 53 - exp;                                    // s = M * 2^-shift, shift >= 53
+  unsigned __int128 P = static_cast<unsigned __int128>(M) * static_cast<unsigned __int128>(m - 1);
+  if (shift >= 128) return 0;
+  return static_cast<int64_t>(P >> shift);
+}
+
+int64_t fade_position_default(int b, int B, int64_t m) {
+  return static_cast<int64_t>((static_cast<__int128>(9) * b * (m - 1)) / (static_cast<__int128>(10) * B));
+}
+
+struct Schedule {
+  std::vector<int32_t> branches;
+  std::vector<int64_t> seg_start, seg_len;
+  int64_t n_active = 0;
+};
+
+// Surviving branches (alpha != 0 and at least one live neuron) and the maximal runs of live
+// neurons inside them, in ascending order.
+void build_schedule(int B, const int64_t* d_b, const float* alpha_eff, const uint8_t* live, Schedule* out) {
+  out->branches.clear();
+  out->seg_start.clear();
+  out->seg_len.clear();
+  out->n_active = 0;
+  int64_t off = 0;
+  for (int b = 0; b < B; ++b) {
+    const int64_t lo = off, hi = off + d_b[b];
+    off = hi;
+    if (alpha_eff[b] == 0.0f) continue;
+    bool any = false;
+    int64_t run = -1;
+    for (int64_t j = lo; j < hi; ++j) {
+      const bool alive = live == nullptr || live[j] != 0;
+      if (alive) {
+        any = true;
+        if (run < 0) run = j;
+      } else if (run >= 0) {
+        out->seg_start.push_back(run);
+        out->seg_len.push_back(j - run);
+        out->n_active += j - run;
+        run = -1;
+      }
+    }
+    if (run >= 0) {
+      out->seg_start.push_back(run);
+      out->seg_len.push_back(hi - run);
+      out->n_active += hi - run;
+    }
+    if (any) out->branches.push_back(b);
+  }
+}
+
+mlpmoe_status_t prune_alpha_host(int B, const float* alpha, const uint8_t* keep, int compensate, float* out) {
+  int K = 0;
+  for (int b = 0; b < B; ++b) K += keep[b] ? 1 : 0;
+  if (K == 0) return MLPMOE_ERR_EMPTY_KEEP_SET;
+  const double c = compensate ? std::sqrt(static_cast<double>(B) / static_cast<double>(K)) : 1.0;
+  for (int b = 0; b < B; ++b) out[b] = keep[b] ? static_cast<float>(c * static_cast<double>(alpha[b])) : 0.0f;
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t check_partition(int64_t d_inter, int B, const int64_t* d_b, int64_t granule) {
+  if (B <= 0 || d_b == nullptr) return MLPMOE_ERR_INVALID_ARG;
+  int64_t sum = 0;
+  for (int b = 0; b < B; ++b) {
+    if (d_b[b] <= 0 || d_b[b] % granule != 0) return MLPMOE_ERR_BAD_PARTITION;
+    sum += d_b[b];
+  }
+  return sum == d_inter ? MLPMOE_OK : MLPMOE_ERR_BAD_PARTITION;
+}
+
+}  // namespace
+
+struct mlpmoe_layer_s {
+  int device = 0, num_sms = 0;
+  int64_t d = 0, I = 0, Ipad_max = 0, max_tokens = 0;
+  int B = 0;
+  mlpmoe_dtype_t dtype = MLPMOE_BF16;
+  int elem_size = 2;
+  std::vector<int64_t> d_b, offs;
+  std::vector<float> alpha_create, alpha_eff;
+  void *Wg_c = nullptr, *Wu_c = nullptr, *Wd_c = nullptr;   // canonical copies, [I x d] each (neuron-major)
+  void *Wgu = nullptr, *WdT = nullptr;                      // packed operands
+  float* scale = nullptr;                                   // [Ipad_max]
+  int32_t* src_row = nullptr;                               // [I] compacted neuron -> original neuron
+  int32_t* row_nnz = nullptr;                               // [3 I]
+  std::vector<int32_t> row_nnz_host;
+  Schedule sched;
+  int64_t Ipad = 0;
+  Workspace* ws = nullptr;
+  void* fade_work = nullptr;
+  float* partial = nullptr;
+  uint32_t* counters = nullptr;
+  int max_splits = 1;
+  uint32_t* status = nullptr;
+  int64_t launches = 0;
+  CUtensorMap tm_wgu, tm_wdt;
+};
+
+namespace {
+
+void free_layer(mlpmoe_layer_s* h) {
+  if (!h) return;
+  cudaFree(h->Wg_c); cudaFree(h->Wu_c); cudaFree(h->Wd_c);
+  cudaFree(h->Wgu); cudaFree(h->WdT);
+  cudaFree(h->scale); cudaFree(h->src_row); cudaFree(h->row_nnz);
+  cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->status);
+  ws_release(h->ws);
+  delete h;
+}
+
+// Recompute liveness, the K-list, the per-neuron scale and the packed operands from the
+// canonical weights and the effective gates.  Synchronises `st`.
+mlpmoe_status_t reschedule(mlpmoe_layer_s* h, cudaStream_t st) {
+  CK(launch_row_nnz(h->Wg_c, h->Wu_c, h->Wd_c, h->row_nnz, h->I, h->d, h->elem_size, st));
+  h->row_nnz_host.resize(3 * h->I);
+  CK(cudaMemcpyAsync(h->row_nnz_host.data(), h->row_nnz, sizeof(int32_t) * 3 * h->I, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  std::vector<uint8_t> live(h->I);
+  for (int64_t j = 0; j < h->I; ++j)
+    live[j] = (h->row_nnz_host[j] > 0 && h->row_nnz_host[h->I + j] > 0 && h->row_nnz_host[2 * h->I + j] > 0) ? 1 : 0;
+  build_schedule(h->B, h->d_b.data(), h->alpha_eff.data(), live.data(), &h->sched);
+  const int64_t n_active = h->sched.n_active;
+  h->Ipad = round_up(n_active > 0 ? n_active : 1, kGroup);
+
+  std::vector<int32_t> src(static_cast<size_t>(n_active > 0 ? n_active : 1));
+  std::vector<float> scale(static_cast<size_t>(h->Ipad), 0.0f);
+  int64_t jj = 0;
+  int b = 0;
+  for (size_t sgi = 0; sgi < h->sched.seg_start.size(); ++sgi) {
+    const int64_t s0 = h->sched.seg_start[sgi], len = h->sched.seg_len[sgi];
+    while (h->offs[b + 1] <= s0) ++b;
+    for (int64_t j = s0; j < s0 + len; ++j, ++jj) {
+      src[jj] = static_cast<int32_t>(j);
+      scale[jj] = h->alpha_eff[b];
+    }
+  }
+  if (n_active > 0) CK(cudaMemcpyAsync(h->src_row, src.data(), sizeof(int32_t) * n_active, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(h->scale, scale.data(), sizeof(float) * h->Ipad, cudaMemcpyHostToDevice, st));
+  CK(launch_gather_gateup(h->Wg_c, h->Wu_c, h->src_row, h->Wgu, n_active, h->Ipad, h->d, h->elem_size, st));
+  CK(launch_gather_down_t(h->Wd_c, h->src_row, h->WdT, n_active, h->Ipad, h->d, h->elem_size, st));
+  CK(cudaStreamSynchronize(st));    // the host vectors above go out of scope
+  if (h->dtype == MLPMOE_BF16) {
+    if (!make_tmap(&h->tm_wgu, h->Wgu, h->d, 2 * h->Ipad, h->d, 256)) return MLPMOE_ERR_CUDA;
+    if (!make_tmap(&h->tm_wdt, h->WdT, h->Ipad, h->d, h->Ipad, 128)) return MLPMOE_ERR_CUDA;
+  }
+  return MLPMOE_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t n, const float* residual,
+                             mlpmoe_dtype_t y_dtype, cudaStream_t st) {
+  if (!h || n < 0) return MLPMOE_ERR_INVALID_ARG;
+  if (n == 0) return MLPMOE_OK;
+  if (!x || !y || n > h->max_tokens || !aligned16(x) || !aligned16(y) || (residual && !aligned16(residual)))
+    return MLPMOE_ERR_INVALID_ARG;
+  if (y_dtype != MLPMOE_FP32 && !(y_dtype == MLPMOE_BF16 && h->dtype == MLPMOE_BF16)) return MLPMOE_ERR_UNSUPPORTED;
+  if (h->dtype == MLPMOE_FP32) {
+    float* H = static_cast<float*>(h->ws->H);
+    CK(launch_simt_gateup(static_cast<const float*>(x), static_cast<const float*>(h->Wgu), h->scale, H, n, h->d, h->Ipad, st));
+    CK(launch_simt_down(H, static_cast<const float*>(h->WdT), residual, static_cast<float*>(y), n, h->d, h->Ipad, st));
+    h->launches += 2;
+    return MLPMOE_OK;
+  }
+  if (n <= kDecodeMaxTokens) {
+    DecodeArgs a;
+    a.npad = n <= 16 ? 16 : (n <= 32 ? 32 : 64);
+    a.tm_w = h->tm_wgu;
+    a.tm_wd = h->tm_wdt;
+    if (!make_tmap(&a.tm_x, x, h->d, n, h->d, a.npad)) return MLPMOE_ERR_CUDA;
+    if (!make_tmap(&a.tm_h, h->ws->H, h->Ipad, n, h->Ipad, a.npad)) return MLPMOE_ERR_CUDA;
+    a.scale = h->scale;
+    a.Hd = h->ws->H;
+    a.partial = h->partial;
+    a.counters = h->counters;
+    a.R = residual;
+    a.Y = y;
+    a.y_bf16 = y_dtype == MLPMOE_BF16;
+    a.n = n; a.d = h->d; a.Ipad = h->Ipad;
+    const int m_blocks = static_cast<int>((h->d + 127) / 128);
+    int splits = h->num_sms / m_blocks;
+    if (splits > h->max_splits) splits = h->max_splits;
+    if (splits > h->Ipad / 64) splits = static_cast<int>(h->Ipad / 64);
+    if (splits < 1) splits = 1;
+    a.splits = splits;
+    a.status = h->status;
+    CK(launch_decode(a, h->num_sms, st));
+    h->launches += 2;
+    return MLPMOE_OK;
+  }
+  TcGateUpArgs g;
+  if (!make_tmap(&g.tm_x, x, h->d, n, h->d, 128)) return MLPMOE_ERR_CUDA;
+  g.tm_w = h->tm_wgu;
+  g.scale = h->scale;
+  g.H = h->ws->H;
+  g.n = n; g.d = h->d; g.Ipad = h->Ipad;
+  g.status = h->status;
+  CK(launch_tc_gateup(g, h->num_sms, st));
+  TcDownArgs dn;
+  if (!make_tmap(&dn.tm_h, h->ws->H, h->Ipad, n, h->Ipad, 128)) return MLPMOE_ERR_CUDA;
+  dn.tm_w = h->tm_wdt;
+  dn.R = residual;
+  dn.Y = y;
+  dn.y_bf16 = y_dtype == MLPMOE_BF16;
+  dn.n = n; dn.d = h->d; dn.Ipad = h->Ipad;
+  dn.status = h->status;
+  CK(launch_tc_down(dn, h->num_sms, st));
+  h->launches += 2;
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t check_stack(const mlpmoe_handle_t* layers, int32_t n_layers, int64_t n) {
+  if (!layers || n_layers <= 0 || n < 0) return MLPMOE_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l) {
+    if (!layers[l]) return MLPMOE_ERR_INVALID_ARG;
+    if (layers[l]->d != layers[0]->d || layers[l]->dtype != layers[0]->dtype) return MLPMOE_ERR_INVALID_ARG;
+    if (n > layers[l]->max_tokens) return MLPMOE_ERR_INVALID_ARG;
+  }
+  return MLPMOE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_inter, int32_t B, const int64_t* d_b,
+                              const void* W_gate, const void* W_up, const void* W_down, const float* alpha,
+                              mlpmoe_dtype_t dtype, mlpmoe_layout_t layout, int64_t max_tokens, void* stream) {
+  if (!out) return MLPMOE_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (d_model <= 0 || d_inter <= 0 || max_tokens <= 0 || !W_gate || !W_up || !W_down) return MLPMOE_ERR_INVALID_ARG;
+  if (dtype != MLPMOE_BF16 && dtype != MLPMOE_FP32) return MLPMOE_ERR_INVALID_ARG;
+  if (layout != MLPMOE_LAYOUT_PAPER && layout != MLPMOE_LAYOUT_LINEAR) return MLPMOE_ERR_INVALID_ARG;
+  mlpmoe_status_t ps = check_partition(d_inter, B, d_b, 16);
+  if (ps != MLPMOE_OK) return ps;
+  if (d_model % 8 != 0) return MLPMOE_ERR_UNSUPPORTED;
+  if (d_inter > (int64_t(1) << 30) || d_model > (int64_t(1) << 30)) return MLPMOE_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  int dev = 0;
+  CK(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  CK(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) return MLPMOE_ERR_UNSUPPORTED;     // kernels are built for sm_100a only
+  CK(tc_gemm_init());
+  CK(decode_init());
+
+  mlpmoe_layer_s* h = new (std::nothrow) mlpmoe_layer_s();
+  if (!h) return MLPMOE_ERR_ALLOC;
+  h->device = dev;
+  h->num_sms = prop.multiProcessorCount;
+  h->d = d_model;
+  h->I = d_inter;
+  h->B = B;
+  h->dtype = dtype;
+  h->elem_size = dtype == MLPMOE_BF16 ? 2 : 4;
+  h->max_tokens = max_tokens;
+  h->Ipad_max = round_up(d_inter, kGroup);
+  h->d_b.assign(d_b, d_b + B);
+  h->offs.resize(B + 1);
+  h->offs[0] = 0;
+  for (int b = 0; b < B; ++b) h->offs[b + 1] = h->offs[b] + d_b[b];
+  h->alpha_create.resize(B);
+  for (int b = 0; b < B; ++b) h->alpha_create[b] = alpha ? alpha[b] : 1.0f;
+  h->alpha_eff = h->alpha_create;
+
+  const size_t es = static_cast<size_t>(h->elem_size);
+  const size_t mat = static_cast<size_t>(d_model) * d_inter * es;
+  const int m_blocks = static_cast<int>((d_model + 127) / 128);
+  h->max_splits = h->num_sms / m_blocks + 1;
+  h->ws = new (std::nothrow) Workspace();
+  bool ok = h->ws != nullptr;
+  if (ok) {
+    h->ws->refs = 1;
+    h->ws->max_tokens = max_tokens;
+    h->ws->Ipad_max = h->Ipad_max;
+    h->ws->d = d_model;
+    h->ws->elem_size = h->elem_size;
+  }
+  ok = ok && cudaMalloc(&h->Wg_c, mat) == cudaSuccess && cudaMalloc(&h->Wu_c, mat) == cudaSuccess &&
+       cudaMalloc(&h->Wd_c, mat) == cudaSuccess &&
+       cudaMalloc(&h->Wgu, static_cast<size_t>(2 * h->Ipad_max) * d_model * es) == cudaSuccess &&
+       cudaMalloc(&h->WdT, static_cast<size_t>(h->Ipad_max) * d_model * es) == cudaSuccess &&
+       cudaMalloc(&h->scale, sizeof(float) * h->Ipad_max) == cudaSuccess &&
+       cudaMalloc(&h->src_row, sizeof(int32_t) * d_inter) == cudaSuccess &&
+       cudaMalloc(&h->row_nnz, sizeof(int32_t) * 3 * d_inter) == cudaSuccess &&
+       cudaMalloc(&h->fade_work, fade_work_bytes(2 * B)) == cudaSuccess &&
+       cudaMalloc(&h->partial, sizeof(float) * static_cast<size_t>(h->max_splits) * d_model * kDecodeMaxTokens) == cudaSuccess &&
+       cudaMalloc(&h->counters, sizeof(uint32_t) * m_blocks * 4) == cudaSuccess &&
+       cudaMalloc(&h->status, sizeof(uint32_t)) == cudaSuccess &&
+       cudaMalloc(&h->ws->H, static_cast<size_t>(max_tokens) * h->Ipad_max * es) == cudaSuccess &&
+       cudaMalloc(&h->ws->xnorm, static_cast<size_t>(max_tokens) * d_model * es) == cudaSuccess &&
+       cudaMalloc(reinterpret_cast<void**>(&h->ws->yres), static_cast<size_t>(max_tokens) * d_model * sizeof(float)) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    free_layer(h);
+    return MLPMOE_ERR_ALLOC;
+  }
+  mlpmoe_status_t rc = MLPMOE_OK;
+  auto fail = [&](mlpmoe_status_t s) { free_layer(h); return s; };
+  if (cudaMemsetAsync(h->counters, 0, sizeof(uint32_t) * m_blocks * 4, st) != cudaSuccess ||
+      cudaMemsetAsync(h->status, 0, sizeof(uint32_t), st) != cudaSuccess)
+    return fail(MLPMOE_ERR_CUDA);
+  // canonical copies: one row of d contiguous weights per intermediate neuron, for all three matrices
+  cudaError_t e;
+  if (layout == MLPMOE_LAYOUT_PAPER) {
+    e = launch_transpose(W_gate, h->Wg_c, d_model, d_inter, h->elem_size, st);
+    if (e == cudaSuccess) e = launch_transpose(W_up, h->Wu_c, d_model, d_inter, h->elem_size, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->Wd_c, W_down, mat, cudaMemcpyDeviceToDevice, st);
+  } else {
+    e = cudaMemcpyAsync(h->Wg_c, W_gate, mat, cudaMemcpyDeviceToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->Wu_c, W_up, mat, cudaMemcpyDeviceToDevice, st);
+    if (e == cudaSuccess) e = launch_transpose(W_down, h->Wd_c, d_model, d_inter, h->elem_size, st);
+  }
+  if (e != cudaSuccess) return fail(MLPMOE_ERR_CUDA);
+  rc = reschedule(h, st);
+  if (rc != MLPMOE_OK) return fail(rc);
+  *out = h;
+  return MLPMOE_OK;
+}
+
+void mlpmoe_destroy(mlpmoe_handle_t h) { free_layer(h); }
+
+mlpmoe_status_t mlpmoe_share_workspace(mlpmoe_handle_t h, mlpmoe_handle_t donor) {
+  if (!h || !donor) return MLPMOE_ERR_INVALID_ARG;
+  if (h->ws == donor->ws) return MLPMOE_OK;
+  const Workspace* w = donor->ws;
+  if (w->elem_size != h->elem_size || w->max_tokens < h->max_tokens || w->Ipad_max < h->Ipad_max || w->d < h->d)
+    return MLPMOE_ERR_INVALID_ARG;
+  ws_release(h->ws);
+  h->ws = donor->ws;
+  h->ws->refs += 1;
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_fade(mlpmoe_handle_t h, const double* s, void* stream) {
+  if (!h) return MLPMOE_ERR_INVALID_ARG;
+  if (s) {
+    for (int b = 0; b < h->B; ++b)
+      if (!(s[b] >= 0.0 && s[b] < 1.0)) return MLPMOE_ERR_BAD_SCHEDULE;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  std::vector<FadeSeg> segs;
+  for (int b = 0; b < h->B; ++b) {
+    const int64_t m = h->d * h->d_b[b];
+    if (s ? (s[b] == 0.0) : (b == 0)) continue;      // the dense backbone / "leave untouched"
+    const int64_t lo = s ? fade_position_exact(s[b], m) : fade_position_default(b, h->B, m);
+    for (int proj = 0; proj < 2; ++proj) {
+      FadeSeg g;
+      g.base = static_cast<char*>(proj == 0 ? h->Wg_c : h->Wu_c) + static_cast<size_t>(h->offs[b]) * h->d * h->elem_size;
+      g.m = m;
+      g.rank = lo;
+      segs.push_back(g);
+    }
+  }
+  CK(launch_fade(segs.data(), static_cast<int>(segs.size()), h->fade_work, h->elem_size, st));
+  CK(cudaStreamSynchronize(st));     // segs is host memory read by an async copy
+  return reschedule(h, st);
+}
+
+mlpmoe_status_t mlpmoe_prune(mlpmoe_handle_t h, const uint8_t* keep, int32_t compensate, void* stream) {
+  if (!h || !keep) return MLPMOE_ERR_INVALID_ARG;
+  std::vector<float> a(h->B);
+  mlpmoe_status_t rc = prune_alpha_host(h->B, h->alpha_create.data(), keep, compensate, a.data());
+  if (rc != MLPMOE_OK) return rc;
+  std::vector<float> saved = h->alpha_eff;
+  h->alpha_eff = a;
+  rc = reschedule(h, static_cast<cudaStream_t>(stream));
+  if (rc != MLPMOE_OK) h->alpha_eff = saved;
+  return rc;
+}
+
+mlpmoe_status_t mlpmoe_prune_first_k(mlpmoe_handle_t h, int32_t K, void* stream) {
+  if (!h) return MLPMOE_ERR_INVALID_ARG;
+  if (K <= 0) return MLPMOE_ERR_EMPTY_KEEP_SET;
+  if (K > h->B) return MLPMOE_ERR_INVALID_ARG;
+  std::vector<uint8_t> keep(h->B);
+  for (int b = 0; b < h->B; ++b) keep[b] = b < K ? 1 : 0;
+  return mlpmoe_prune(h, keep.data(), 1, stream);
+}
+
+mlpmoe_status_t mlpmoe_forward(mlpmoe_handle_t h, const void* x, void* y, int64_t n_tokens, void* stream) {
+  return forward_impl(h, x, y, n_tokens, nullptr, MLPMOE_FP32, static_cast<cudaStream_t>(stream));
+}
+
+mlpmoe_status_t mlpmoe_forward_ex(mlpmoe_handle_t h, const void* x, void* y, int64_t n_tokens, const float* residual,
+                                  mlpmoe_dtype_t y_dtype, void* stream) {
+  return forward_impl(h, x, y, n_tokens, residual, y_dtype, static_cast<cudaStream_t>(stream));
+}
+
+mlpmoe_status_t mlpmoe_forward_host(mlpmoe_handle_t h, const void* x_host, float* y_host, int64_t n, void* stream) {
+  if (!h || n < 0) return MLPMOE_ERR_INVALID_ARG;
+  if (n == 0) return MLPMOE_OK;
+  if (!x_host || !y_host || n > h->max_tokens) return MLPMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CK(cudaMemcpyAsync(h->ws->xnorm, x_host, static_cast<size_t>(n) * h->d * h->elem_size, cudaMemcpyHostToDevice, st));
+  mlpmoe_status_t rc = forward_impl(h, h->ws->xnorm, h->ws->yres, n, nullptr, MLPMOE_FP32, st);
+  if (rc != MLPMOE_OK) return rc;
+  CK(cudaMemcpyAsync(y_host, h->ws->yres, static_cast<size_t>(n) * h->d * sizeof(float), cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_rmsnorm(const float* x, void* r, int64_t n_tokens, int64_t d_model, float eps,
+                               mlpmoe_dtype_t out_dtype, void* stream) {
+  if (n_tokens < 0 || d_model <= 0 || d_model % 4 != 0) return MLPMOE_ERR_INVALID_ARG;
+  if (n_tokens == 0) return MLPMOE_OK;
+  if (!x || !r || !aligned16(x) || !aligned16(r)) return MLPMOE_ERR_INVALID_ARG;
+  CK(launch_rmsnorm(x, r, n_tokens, d_model, eps, out_dtype == MLPMOE_BF16 ? 2 : 4, static_cast<cudaStream_t>(stream)));
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_layers, float* x, int64_t n, float eps,
+                                     void* stream) {
+  mlpmoe_status_t rc = check_stack(layers, n_layers, n);
+  if (rc != MLPMOE_OK) return rc;
+  if (n == 0) return MLPMOE_OK;
+  if (!x || !aligned16(x)) return MLPMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  for (int l = 0; l < n_layers; ++l) {
+    mlpmoe_layer_s* h = layers[l];
+    CK(launch_rmsnorm(x, h->ws->xnorm, n, h->d, eps, h->elem_size, st));
+    h->launches += 1;
+    rc = forward_impl(h, h->ws->xnorm, x, n, x, MLPMOE_FP32, st);
+    if (rc != MLPMOE_OK) return rc;
+  }
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_stack_forward_host(const mlpmoe_handle_t* layers, int32_t n_layers, const float* x_host,
+                                          float* y_host, int64_t n, float eps, void* stream) {
+  mlpmoe_status_t rc = check_stack(layers, n_layers, n);
+  if (rc != MLPMOE_OK) return rc;
+  if (n == 0) return MLPMOE_OK;
+  if (!x_host || !y_host) return MLPMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  mlpmoe_layer_s* h0 = layers[0];
+  const size_t bytes = static_cast<size_t>(n) * h0->d * sizeof(float);
+  CK(cudaMemcpyAsync(h0->ws->yres, x_host, bytes, cudaMemcpyHostToDevice, st));
+  rc = mlpmoe_stack_forward(layers, n_layers, h0->ws->yres, n, eps, stream);
+  if (rc != MLPMOE_OK) return rc;
+  CK(cudaMemcpyAsync(y_host, h0->ws->yres, bytes, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_get_klist(mlpmoe_handle_t h, int32_t* branches, int32_t* n_branches, int64_t* seg_start,
+                                 int64_t* seg_len, int32_t* n_segs) {
+  if (!h) return MLPMOE_ERR_INVALID_ARG;
+  const Schedule& s = h->sched;
+  if (branches) std::memcpy(branches, s.branches.data(), sizeof(int32_t) * s.branches.size());
+  if (n_branches) *n_branches = static_cast<int32_t>(s.branches.size());
+  if (seg_start) std::memcpy(seg_start, s.seg_start.data(), sizeof(int64_t) * s.seg_start.size());
+  if (seg_len) std::memcpy(seg_len, s.seg_len.data(), sizeof(int64_t) * s.seg_len.size());
+  if (n_segs) *n_segs = static_cast<int32_t>(s.seg_start.size());
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_get_alpha(mlpmoe_handle_t h, float* alpha) {
+  if (!h || !alpha) return MLPMOE_ERR_INVALID_ARG;
+  std::memcpy(alpha, h->alpha_eff.data(), sizeof(float) * h->B);
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_get_active_neurons(mlpmoe_handle_t h, int64_t* n_active) {
+  if (!h || !n_active) return MLPMOE_ERR_INVALID_ARG;
+  *n_active = h->sched.n_active;
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_nnz(mlpmoe_handle_t h, int64_t* nnz_gate, int64_t* nnz_up, int64_t* nnz_down) {
+  if (!h) return MLPMOE_ERR_INVALID_ARG;
+  // row_nnz_host is refreshed by every reschedule (create, fade, prune), the only calls that change weights
+  int64_t* outs[3] = {nnz_gate, nnz_up, nnz_down};
+  for (int which = 0; which < 3; ++which) {
+    if (!outs[which]) continue;
+    for (int b = 0; b < h->B; ++b) {
+      int64_t c = 0;
+      for (int64_t j = h->offs[b]; j < h->offs[b + 1]; ++j) c += h->row_nnz_host[which * h->I + j];
+      outs[which][b] = c;
+    }
+  }
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_get_weights(mlpmoe_handle_t h, void* W_gate, void* W_up, void* W_down, void* stream) {
+  if (!h) return MLPMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (W_gate) CK(launch_transpose(h->Wg_c, W_gate, h->I, h->d, h->elem_size, st));
+  if (W_up) CK(launch_transpose(h->Wu_c, W_up, h->I, h->d, h->elem_size, st));
+  if (W_down)
+    CK(cudaMemcpyAsync(W_down, h->Wd_c, static_cast<size_t>(h->I) * h->d * h->elem_size, cudaMemcpyDeviceToDevice, st));
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_get_status(mlpmoe_handle_t h) {
+  if (!h) return MLPMOE_ERR_INVALID_ARG;
+  uint32_t w = 0;
+  CK(cudaDeviceSynchronize());
+  CK(cudaMemcpy(&w, h->status, sizeof(w), cudaMemcpyDeviceToHost));
+  return w == kStatusOk ? MLPMOE_OK : MLPMOE_ERR_DEVICE_TIMEOUT;
+}
+
+mlpmoe_status_t mlpmoe_get_launch_count(mlpmoe_handle_t h, int64_t* launches) {
+  if (!h || !launches) return MLPMOE_ERR_INVALID_ARG;
+  *launches = h->launches;
+  return MLPMOE_OK;
+}
+
+const char* mlpmoe_status_string(mlpmoe_status_t s) {
+  switch (s) {
+    case MLPMOE_OK: return "ok";
+    case MLPMOE_ERR_INVALID_ARG: return "invalid argument";
+    case MLPMOE_ERR_BAD_PARTITION: return "bad partition of d_inter";
+    case MLPMOE_ERR_EMPTY_KEEP_SET: return "empty keep set";
+    case MLPMOE_ERR_BAD_SCHEDULE: return "sparsity ratio outside [0, 1)";
+    case MLPMOE_ERR_UNSUPPORTED: return "unsupported shape, dtype or device";
+    case MLPMOE_ERR_ALLOC: return "allocation failed";
+    case MLPMOE_ERR_CUDA: return "CUDA call failed";
+    case MLPMOE_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+  }
+  return "unknown status";
+}
+
+// ---- host-only helpers ------------------------------------------------------
+mlpmoe_status_t mlpmoe_host_fade_position(double s, int64_t m, int64_t* lo) {
+  if (!lo || m <= 0) return MLPMOE_ERR_INVALID_ARG;
+  if (!(s >= 0.0 && s < 1.0)) return MLPMOE_ERR_BAD_SCHEDULE;
+  *lo = fade_position_exact(s, m);
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_host_fade_position_default(int32_t b, int32_t B, int64_t m, int64_t* lo) {
+  if (!lo || m <= 0 || B <= 0 || b < 0 || b >= B) return MLPMOE_ERR_INVALID_ARG;
+  *lo = fade_position_default(b, B, m);
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_host_prune_alpha(int32_t B, const float* alpha, const uint8_t* keep, int32_t compensate,
+                                        float* alpha_eff) {
+  if (B <= 0 || !alpha || !keep || !alpha_eff) return MLPMOE_ERR_INVALID_ARG;
+  return prune_alpha_host(B, alpha, keep, compensate, alpha_eff);
+}
+
+mlpmoe_status_t mlpmoe_host_schedule(int32_t B, const int64_t* d_b, const float* alpha_eff, const uint8_t* live,
+                                     int32_t* branches, int32_t* n_branches, int64_t* seg_start, int64_t* seg_len,
+                                     int32_t* n_segs, int64_t* n_active) {
+  if (B <= 0 || !d_b || !alpha_eff) return MLPMOE_ERR_INVALID_ARG;
+  int64_t I = 0;
+  for (int b = 0; b < B; ++b) {
+    if (d_b[b] <= 0) return MLPMOE_ERR_BAD_PARTITION;
+    I += d_b[b];
+  }
+  Schedule s;
+  build_schedule(B, d_b, alpha_eff, live, &s);
+  if (branches) std::memcpy(branches, s.branches.data(), sizeof(int32_t) * s.branches.size());
+  if (n_branches) *n_branches = static_cast<int32_t>(s.branches.size());
+  if (seg_start) std::memcpy(seg_start, s.seg_start.data(), sizeof(int64_t) * s.seg_start.size());
+  if (seg_len) std::memcpy(seg_len, s.seg_len.data(), sizeof(int64_t) * s.seg_len.size());
+  if (n_segs) *n_segs = static_cast<int32_t>(s.seg_start.size());
+  if (n_active) *n_active = s.n_active;
+  (void)I;
+  return MLPMOE_OK;
+}
+
+}  // extern "C"

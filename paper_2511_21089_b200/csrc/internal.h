@@ -1,0 +1,93 @@
+// Internal launch interface between the C-ABI host code and the kernel files.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mlpmoe {
+
+constexpr int kGroup = 128;      // neurons per interleaved gate|up group in the packed operand
+constexpr int kDecodeMaxTokens = 64;
+
+// Device status word values (written by kernels whose bounded waits run out).
+constexpr uint32_t kStatusOk = 0;
+constexpr uint32_t kStatusTimeout = 1;
+
+// ------------------------------------------------------------------ pack.cu --
+// dst[c * rows + r] = src[r * cols + c]
+cudaError_t launch_transpose(const void* src, void* dst, int64_t rows, int64_t cols, int elem_size, cudaStream_t st);
+// Packed gate|up operand: rows [2*kGroup*q, +kGroup) = gate rows of compacted neurons [kGroup*q, +kGroup),
+// next kGroup rows = their up rows; each row d contiguous elements.  Rows past n_active are zero.
+cudaError_t launch_gather_gateup(const void* Wg_c, const void* Wu_c, const int32_t* src_row, void* Wgu,
+                                 int64_t n_active, int64_t n_active_pad, int64_t d, int elem_size, cudaStream_t st);
+// Packed down operand, K-major: WdT[m * n_active_pad + j'] = Wd_c[src_row[j'] * d + m]; columns past n_active zero.
+cudaError_t launch_gather_down_t(const void* Wd_c, const int32_t* src_row, void* WdT, int64_t n_active,
+                                 int64_t n_active_pad, int64_t d, int elem_size, cudaStream_t st);
+// Per neuron row: non-zero counts of the gate, up and down rows: out[0*I + j], out[1*I + j], out[2*I + j].
+cudaError_t launch_row_nnz(const void* Wg_c, const void* Wu_c, const void* Wd_c, int32_t* out, int64_t I, int64_t d,
+                           int elem_size, cudaStream_t st);
+
+// Fade: exact rank selection on magnitude bit patterns, then masking (Section 3.2).
+struct FadeSeg {
+  void* base;      // first element of the slice (contiguous m elements)
+  int64_t m;       // number of elements
+  int64_t rank;    // 0-based rank lo of the threshold order statistic
+};
+// work: device scratch of fade_work_bytes(nseg) bytes.  Zeroes every element with |w| <= (rank-th smallest |w|).
+size_t fade_work_bytes(int nseg);
+cudaError_t launch_fade(const FadeSeg* segs_host, int nseg, void* work, int elem_size, cudaStream_t st);
+
+// r = x / sqrt(mean(x^2) + eps), out bf16 (elem_size 2) or fp32 (4).
+cudaError_t launch_rmsnorm(const float* x, void* r, int64_t n, int64_t d, float eps, int out_elem_size, cudaStream_t st);
+
+// ------------------------------------------------------------- simt_gemm.cu --
+// fp32 path.  H[n x ldh] = silu(X Wg'^T) * (X Wu'^T) * scale, Wgu packed as above.
+cudaError_t launch_simt_gateup(const float* X, const float* Wgu, const float* scale, float* H, int64_t n, int64_t d,
+                               int64_t n_active_pad, cudaStream_t st);
+// Y[n x d] = (R +) H[n x K] * WdT[d x K]^T
+cudaError_t launch_simt_down(const float* H, const float* WdT, const float* R, float* Y, int64_t n, int64_t d,
+                             int64_t K, cudaStream_t st);
+
+// --------------------------------------------------------------- tc_gemm.cu --
+struct TcGateUpArgs {
+  CUtensorMap tm_x;     // X   [n x d]            bf16, box 64 x 128, 128B swizzle
+  CUtensorMap tm_w;     // Wgu [2*Ipad x d]       bf16, box 64 x 256
+  const float* scale;   // [Ipad]
+  void* H;              // [n x Ipad] bf16
+  int64_t n, d, Ipad;
+  uint32_t* status;
+};
+struct TcDownArgs {
+  CUtensorMap tm_h;     // H   [n x Ipad]         bf16, box 64 x 128
+  CUtensorMap tm_w;     // WdT [d x Ipad]         bf16, box 64 x 128
+  const float* R;       // optional fp32 residual [n x d]
+  void* Y;              // [n x d] fp32 or bf16
+  int y_bf16;
+  int64_t n, d, Ipad;
+  uint32_t* status;
+};
+cudaError_t launch_tc_gateup(const TcGateUpArgs& a, int num_sms, cudaStream_t st);
+cudaError_t launch_tc_down(const TcDownArgs& a, int num_sms, cudaStream_t st);
+cudaError_t tc_gemm_init();   // opt in to the large dynamic shared memory sizes (once per process)
+
+// ---------------------------------------------------------------- decode.cu --
+struct DecodeArgs {
+  CUtensorMap tm_w;     // Wgu [2*Ipad x d]  box 64 x 64
+  CUtensorMap tm_x;     // X   [n x d]       box 64 x npad
+  CUtensorMap tm_wd;    // WdT [d x Ipad]    box 64 x 128
+  CUtensorMap tm_h;     // Hd  [n x Ipad]    box 64 x npad
+  const float* scale;
+  void* Hd;             // [n x Ipad] bf16 workspace
+  float* partial;       // [splits x d x npad] fp32 workspace
+  uint32_t* counters;   // [d / 128] arrival counters, zero between calls
+  const float* R;
+  void* Y;
+  int y_bf16;
+  int64_t n, d, Ipad;
+  int npad, splits;
+  uint32_t* status;
+};
+cudaError_t launch_decode(const DecodeArgs& a, int num_sms, cudaStream_t st);
+cudaError_t decode_init();
+
+}  // namespace mlpmoe

@@ -1,0 +1,307 @@
+// Set-up kernels: weight packer (slice / transpose / interleave, Section 3.1), Fractal Fade
+// (exact rank selection + masking, Section 3.2), per-neuron non-zero counts for the scheduler,
+// and the RMSNorm helper of the stack harness.  All HBM-bound copies.
+#include "internal.h"
+
+namespace mlpmoe {
+namespace {
+
+// ------------------------------------------------------------- transpose ----
+template <typename T>
+__global__ void transpose_kernel(const T* __restrict__ src, T* __restrict__ dst, int64_t rows, int64_t cols) {
+  __shared__ T tile[32][33];
+  const int64_t c0 = static_cast<int64_t>(blockIdx.x) * 32, r0 = static_cast<int64_t>(blockIdx.y) * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int64_t r = r0 + i, c = c0 + threadIdx.x;
+    if (r < rows && c < cols) tile[i][threadIdx.x] = src[r * cols + c];
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int64_t c = c0 + i, r = r0 + threadIdx.x;
+    if (r < rows && c < cols) dst[c * rows + r] = tile[threadIdx.x][i];
+  }
+}
+
+// ------------------------------------------------------ gate|up gather ------
+// One block per packed row; 16-byte vectors (d * elem_size is a multiple of 16).
+__global__ void gather_gateup_kernel(const uint4* __restrict__ Wg_c, const uint4* __restrict__ Wu_c,
+                                     const int32_t* __restrict__ src_row, uint4* __restrict__ Wgu, int64_t n_active,
+                                     int64_t row_vecs) {
+  const int64_t r = blockIdx.x;
+  const int64_t q = r / (2 * kGroup);
+  const int within = static_cast<int>(r % (2 * kGroup));
+  const bool is_up = within >= kGroup;
+  const int64_t j = q * kGroup + (within % kGroup);
+  uint4* out = Wgu + r * row_vecs;
+  if (j < n_active) {
+    const uint4* in = (is_up ? Wu_c : Wg_c) + static_cast<int64_t>(src_row[j]) * row_vecs;
+    for (int64_t v = threadIdx.x; v < row_vecs; v += blockDim.x) out[v] = in[v];
+  } else {
+    for (int64_t v = threadIdx.x; v < row_vecs; v += blockDim.x) out[v] = make_uint4(0, 0, 0, 0);
+  }
+}
+
+// -------------------------------------------------- down gather+transpose ---
+template <typename T>
+__global__ void gather_down_t_kernel(const T* __restrict__ Wd_c, const int32_t* __restrict__ src_row, T* __restrict__ WdT,
+                                     int64_t n_active, int64_t n_active_pad, int64_t d) {
+  __shared__ T tile[32][33];
+  const int64_t j0 = static_cast<int64_t>(blockIdx.x) * 32, m0 = static_cast<int64_t>(blockIdx.y) * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int64_t j = j0 + i, m = m0 + threadIdx.x;
+    T v = T(0);
+    if (j < n_active && m < d) v = Wd_c[static_cast<int64_t>(src_row[j]) * d + m];
+    tile[i][threadIdx.x] = v;
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int64_t m = m0 + i, j = j0 + threadIdx.x;
+    if (m < d && j < n_active_pad) WdT[m * n_active_pad + j] = tile[threadIdx.x][i];
+  }
+}
+
+// ------------------------------------------------------------ row nnz -------
+template <typename T>
+__device__ __forceinline__ bool is_nonzero(T v);
+template <>
+__device__ __forceinline__ bool is_nonzero<uint16_t>(uint16_t v) { return (v & 0x7FFFu) != 0; }
+template <>
+__device__ __forceinline__ bool is_nonzero<uint32_t>(uint32_t v) { return (v & 0x7FFFFFFFu) != 0; }
+
+// One warp per (matrix, neuron row).
+template <typename T>
+__global__ void row_nnz_kernel(const T* __restrict__ Wg_c, const T* __restrict__ Wu_c, const T* __restrict__ Wd_c,
+                               int32_t* __restrict__ out, int64_t I, int64_t d) {
+  const int64_t w = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) / 32;
+  const int lane = threadIdx.x % 32;
+  if (w >= 3 * I) return;
+  const int which = static_cast<int>(w / I);
+  const int64_t j = w % I;
+  const T* row = (which == 0 ? Wg_c : which == 1 ? Wu_c : Wd_c) + j * d;
+  int cnt = 0;
+  for (int64_t k = lane; k < d; k += 32) cnt += is_nonzero<T>(row[k]) ? 1 : 0;
+  for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
+  if (lane == 0) out[w] = cnt;
+}
+
+// --------------------------------------------------------------- Fade -------
+// Keys: magnitude bit patterns as 32-bit integers (order of non-negative floats equals the
+// order of their bit patterns).  bf16 magnitudes are placed in the upper half so that the
+// same digit positions serve both types.
+template <typename T>
+__device__ __forceinline__ uint32_t mag_key(T v);
+template <>
+__device__ __forceinline__ uint32_t mag_key<uint16_t>(uint16_t v) { return static_cast<uint32_t>(v & 0x7FFFu) << 16; }
+template <>
+__device__ __forceinline__ uint32_t mag_key<uint32_t>(uint32_t v) { return v & 0x7FFFFFFFu; }
+
+struct FadeSegDev {
+  void* base;
+  int64_t m;
+  int64_t rank;
+};
+struct FadeState {          // per segment
+  uint32_t prefix;          // digits fixed so far (upper bits of the threshold key)
+  uint32_t pad;
+  int64_t remaining;        // rank among the elements that match the prefix
+  uint32_t hist[256];
+};
+
+__global__ void fade_init_kernel(const FadeSegDev* segs, FadeState* st, int nseg) {
+  const int s = blockIdx.x;
+  if (s >= nseg) return;
+  if (threadIdx.x == 0) {
+    st[s].prefix = 0;
+    st[s].remaining = segs[s].rank;
+  }
+  for (int i = threadIdx.x; i < 256; i += blockDim.x) st[s].hist[i] = 0;
+}
+
+// Histogram of digit `pass` (8 bits, most significant first) over elements matching the prefix.
+template <typename T>
+__global__ void fade_hist_kernel(const FadeSegDev* segs, FadeState* st, int pass) {
+  __shared__ uint32_t h[256];
+  const int s = blockIdx.y;
+  for (int i = threadIdx.x; i < 256; i += blockDim.x) h[i] = 0;
+  __syncthreads();
+  const T* base = static_cast<const T*>(segs[s].base);
+  const int64_t m = segs[s].m;
+  const int shift = 24 - 8 * pass;
+  const uint32_t himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+  const uint32_t prefix = st[s].prefix;
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < m;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const uint32_t key = mag_key<T>(base[i]);
+    if ((key & himask) == prefix) atomicAdd(&h[(key >> shift) & 0xFFu], 1u);
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < 256; i += blockDim.x)
+    if (h[i]) atomicAdd(&st[s].hist[i], h[i]);
+}
+
+// Pick the digit whose bin holds the wanted rank; fix it in the prefix; clear the histogram.
+__global__ void fade_select_kernel(FadeState* st, int pass) {
+  const int s = blockIdx.x;
+  if (threadIdx.x == 0) {
+    const int shift = 24 - 8 * pass;
+    int64_t rem = st[s].remaining;
+    int digit = 255;
+    for (int b = 0; b < 256; ++b) {
+      const int64_t c = st[s].hist[b];
+      if (rem < c) { digit = b; break; }
+      rem -= c;
+    }
+    st[s].prefix |= static_cast<uint32_t>(digit) << shift;
+    st[s].remaining = rem;
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < 256; i += blockDim.x) st[s].hist[i] = 0;
+}
+
+// Zero every element whose magnitude key is <= the threshold key (keeps the sign bit, as a
+// multiplication by a 0/1 mask does).
+template <typename T>
+__global__ void fade_mask_kernel(const FadeSegDev* segs, const FadeState* st) {
+  const int s = blockIdx.y;
+  T* base = static_cast<T*>(segs[s].base);
+  const int64_t m = segs[s].m;
+  const uint32_t thr = st[s].prefix;
+  constexpr T sign = static_cast<T>(T(1) << (8 * sizeof(T) - 1));
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < m;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const T v = base[i];
+    if (mag_key<T>(v) <= thr) base[i] = v & sign;
+  }
+}
+
+// ------------------------------------------------------------- RMSNorm ------
+__device__ __forceinline__ uint16_t f32_to_bf16_rn(float f) {
+  uint32_t u = __float_as_uint(f);
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return static_cast<uint16_t>(u >> 16);
+}
+
+template <bool OUT_BF16>
+__global__ void rmsnorm_kernel(const float* __restrict__ x, void* __restrict__ r, int64_t n, int64_t d, float eps) {
+  const int64_t t = blockIdx.x;
+  const float4* row = reinterpret_cast<const float4*>(x + t * d);
+  const int64_t nv = d / 4;
+  float ss = 0.f;
+  for (int64_t v = threadIdx.x; v < nv; v += blockDim.x) {
+    const float4 a = row[v];
+    ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+  }
+  __shared__ float red[32];
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+  if (threadIdx.x % 32 == 0) red[threadIdx.x / 32] = ss;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float v = threadIdx.x < blockDim.x / 32 ? red[threadIdx.x] : 0.f;
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    if (threadIdx.x == 0) red[0] = v;
+  }
+  __syncthreads();
+  const float inv = 1.0f / sqrtf(red[0] / static_cast<float>(d) + eps);
+  for (int64_t v = threadIdx.x; v < nv; v += blockDim.x) {
+    const float4 a = row[v];
+    if (OUT_BF16) {
+      uint2 o;
+      o.x = static_cast<uint32_t>(f32_to_bf16_rn(a.x * inv)) | (static_cast<uint32_t>(f32_to_bf16_rn(a.y * inv)) << 16);
+      o.y = static_cast<uint32_t>(f32_to_bf16_rn(a.z * inv)) | (static_cast<uint32_t>(f32_to_bf16_rn(a.w * inv)) << 16);
+      reinterpret_cast<uint2*>(static_cast<uint16_t*>(r) + t * d)[v] = o;
+    } else {
+      reinterpret_cast<float4*>(static_cast<float*>(r) + t * d)[v] = make_float4(a.x * inv, a.y * inv, a.z * inv, a.w * inv);
+    }
+  }
+}
+
+inline unsigned cdiv(int64_t a, int64_t b) { return static_cast<unsigned>((a + b - 1) / b); }
+
+}  // namespace
+
+cudaError_t launch_transpose(const void* src, void* dst, int64_t rows, int64_t cols, int elem_size, cudaStream_t st) {
+  if (rows == 0 || cols == 0) return cudaSuccess;
+  dim3 grid(cdiv(cols, 32), cdiv(rows, 32)), block(32, 8);
+  if (elem_size == 2)
+    transpose_kernel<uint16_t><<<grid, block, 0, st>>>(static_cast<const uint16_t*>(src), static_cast<uint16_t*>(dst), rows, cols);
+  else
+    transpose_kernel<uint32_t><<<grid, block, 0, st>>>(static_cast<const uint32_t*>(src), static_cast<uint32_t*>(dst), rows, cols);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather_gateup(const void* Wg_c, const void* Wu_c, const int32_t* src_row, void* Wgu, int64_t n_active,
+                                 int64_t n_active_pad, int64_t d, int elem_size, cudaStream_t st) {
+  if (n_active_pad == 0) return cudaSuccess;
+  const int64_t row_vecs = d * elem_size / 16;
+  gather_gateup_kernel<<<static_cast<unsigned>(2 * n_active_pad), 128, 0, st>>>(
+      static_cast<const uint4*>(Wg_c), static_cast<const uint4*>(Wu_c), src_row, static_cast<uint4*>(Wgu), n_active, row_vecs);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather_down_t(const void* Wd_c, const int32_t* src_row, void* WdT, int64_t n_active,
+                                 int64_t n_active_pad, int64_t d, int elem_size, cudaStream_t st) {
+  if (n_active_pad == 0) return cudaSuccess;
+  dim3 grid(cdiv(n_active_pad, 32), cdiv(d, 32)), block(32, 8);
+  if (elem_size == 2)
+    gather_down_t_kernel<uint16_t><<<grid, block, 0, st>>>(static_cast<const uint16_t*>(Wd_c), src_row,
+                                                           static_cast<uint16_t*>(WdT), n_active, n_active_pad, d);
+  else
+    gather_down_t_kernel<uint32_t><<<grid, block, 0, st>>>(static_cast<const uint32_t*>(Wd_c), src_row,
+                                                           static_cast<uint32_t*>(WdT), n_active, n_active_pad, d);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_row_nnz(const void* Wg_c, const void* Wu_c, const void* Wd_c, int32_t* out, int64_t I, int64_t d,
+                           int elem_size, cudaStream_t st) {
+  const int64_t warps = 3 * I;
+  const unsigned blocks = cdiv(warps * 32, 256);
+  if (elem_size == 2)
+    row_nnz_kernel<uint16_t><<<blocks, 256, 0, st>>>(static_cast<const uint16_t*>(Wg_c), static_cast<const uint16_t*>(Wu_c),
+                                                     static_cast<const uint16_t*>(Wd_c), out, I, d);
+  else
+    row_nnz_kernel<uint32_t><<<blocks, 256, 0, st>>>(static_cast<const uint32_t*>(Wg_c), static_cast<const uint32_t*>(Wu_c),
+                                                     static_cast<const uint32_t*>(Wd_c), out, I, d);
+  return cudaGetLastError();
+}
+
+size_t fade_work_bytes(int nseg) { return static_cast<size_t>(nseg) * (sizeof(FadeSegDev) + sizeof(FadeState)); }
+
+cudaError_t launch_fade(const FadeSeg* segs_host, int nseg, void* work, int elem_size, cudaStream_t st) {
+  if (nseg == 0) return cudaSuccess;
+  static_assert(sizeof(FadeSeg) == sizeof(FadeSegDev), "segment records must match");
+  FadeSegDev* segs = static_cast<FadeSegDev*>(work);
+  FadeState* state = reinterpret_cast<FadeState*>(segs + nseg);
+  cudaError_t e = cudaMemcpyAsync(segs, segs_host, sizeof(FadeSegDev) * nseg, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return e;
+  int64_t max_m = 0;
+  for (int i = 0; i < nseg; ++i) max_m = segs_host[i].m > max_m ? segs_host[i].m : max_m;
+  unsigned bx = cdiv(max_m, 256 * 16);
+  if (bx > 1024) bx = 1024;
+  if (bx < 1) bx = 1;
+  dim3 grid(bx, nseg);
+  fade_init_kernel<<<nseg, 256, 0, st>>>(segs, state, nseg);
+  const int passes = elem_size == 2 ? 2 : 4;   // bf16 keys carry 15 significant bits in the upper half
+  for (int p = 0; p < passes; ++p) {
+    if (elem_size == 2)
+      fade_hist_kernel<uint16_t><<<grid, 256, 0, st>>>(segs, state, p);
+    else
+      fade_hist_kernel<uint32_t><<<grid, 256, 0, st>>>(segs, state, p);
+    fade_select_kernel<<<nseg, 256, 0, st>>>(state, p);
+  }
+  if (elem_size == 2)
+    fade_mask_kernel<uint16_t><<<grid, 256, 0, st>>>(segs, state);
+  else
+    fade_mask_kernel<uint32_t><<<grid, 256, 0, st>>>(segs, state);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rmsnorm(const float* x, void* r, int64_t n, int64_t d, float eps, int out_elem_size, cudaStream_t st) {
+  if (n == 0) return cudaSuccess;
+  if (out_elem_size == 2)
+    rmsnorm_kernel<true><<<static_cast<unsigned>(n), 256, 0, st>>>(x, r, n, d, eps);
+  else
+    rmsnorm_kernel<false><<<static_cast<unsigned>(n), 256, 0, st>>>(x, r, n, d, eps);
+  return cudaGetLastError();
+}
+
+}  // namespace mlpmoe

@@ -1,0 +1,283 @@
+// Prefill path on the 5th-generation tensor cores (sm_100a): two persistent, warp-specialised
+// GEMM kernels with bf16 operands staged by TMA into 128-byte-swizzled shared memory, tcgen05.mma
+// accumulating in fp32 in tensor memory, and a double-buffered accumulator so that the epilogue
+// of one tile runs under the MMAs of the next.
+//
+//   gate|up  (Section 3.1, inner bracket):   one 128 x 256 accumulator holds gate (columns 0..127)
+//            and up (columns 128..255) of the same 128 neurons; the epilogue computes
+//            H = bf16( silu(gate) * up * scale ), scale[j] = effective alpha of neuron j's branch.
+//   down     (Section 3.1, outer product and branch sum): Y = (R +) H * WdT^T with the K loop
+//            running over every surviving neuron of every surviving branch in one accumulator.
+//
+// Warp roles (192 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM owner + MMA issuer
+// (one lane), warps 2..5 = epilogue (TMEM lane quadrant = warp index mod 4).
+#include <cuda_bf16.h>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace mlpmoe {
+namespace {
+
+using namespace ptx;
+
+constexpr int BM = 128;        // rows of the A tile = UMMA M
+constexpr int BK = 64;         // K elements per stage: one 128-byte swizzled row of bf16
+constexpr int UMMA_K = 16;
+constexpr int NUM_THREADS = 192;
+
+enum { EPI_SWIGLU = 0, EPI_OUT = 1 };
+
+template <int BN, int STAGES>
+struct Cfg {
+  static constexpr int A_BYTES = BM * BK * 2;
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+  static constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;   // barriers + slack for 1024-byte alignment
+  static constexpr int TMEM_COLS = 2 * BN;                      // two accumulator buffers
+};
+
+struct EpiArgs {
+  const float* scale;   // EPI_SWIGLU
+  const float* R;       // EPI_OUT, optional
+  void* out;            // H (bf16) or Y (fp32 / bf16)
+  int64_t rows;         // valid rows (tokens)
+  int64_t cols;         // valid output columns (EPI_OUT: d; EPI_SWIGLU: Ipad)
+  int64_t ld;           // output row pitch in elements
+  int out_bf16;         // EPI_OUT only
+  uint32_t* status;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int BN, int STAGES, int EPI>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const EpiArgs ep,
+               int num_m_blocks, int num_n_blocks, int num_k_blocks) {
+  using C = Cfg<BN, STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + C::BAR_OFFSET);
+  uint64_t* empty_bar = full_bar + STAGES;
+  uint64_t* tfull_bar = empty_bar + STAGES;
+  uint64_t* tempty_bar = tfull_bar + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&tfull_bar[a], 1);
+      mbar_init(&tempty_bar[a], 4);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, C::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int num_tiles = num_m_blocks * num_n_blocks;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      prefetch_tensormap(&tm_a);
+      prefetch_tensormap(&tm_b);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        const int m_blk = tile % num_m_blocks, n_blk = tile / num_m_blocks;
+        for (int kb = 0; kb < num_k_blocks; ++kb) {
+          if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+          uint8_t* sa = smem + stage * C::STAGE_BYTES;
+          mbar_expect_tx(&full_bar[stage], C::STAGE_BYTES);
+          tma_load_2d(sa, &tm_a, kb * BK, m_blk * BM, &full_bar[stage]);
+          tma_load_2d(sa + C::A_BYTES, &tm_b, kb * BK, n_blk * BN, &full_bar[stage]);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16_f32(BM, BN);
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        if (!mbar_wait_bounded(&tempty_bar[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+        for (int kb = 0; kb < num_k_blocks; ++kb) {
+          if (!mbar_wait_bounded(&full_bar[stage], phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + stage * C::STAGE_BYTES);
+          const uint64_t a_desc = make_desc_sw128_kmajor(sa);
+          const uint64_t b_desc = make_desc_sw128_kmajor(sa + C::A_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // advancing 16 elements along K inside the swizzled row = +32 bytes = +2 in the address field
+            umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(&empty_bar[stage]);       // stage is free once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(&tfull_bar[acc]);           // accumulator complete
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int quad = warp % 4;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+      const int m_blk = tile % num_m_blocks, n_blk = tile / num_m_blocks;
+      bool ok = mbar_wait_bounded(&tfull_bar[acc], acc_phase, abort_flag);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int64_t row = static_cast<int64_t>(m_blk) * BM + quad * 32 + lane;
+      const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * BN) + (static_cast<uint32_t>(quad * 32) << 16);
+      if (EPI == EPI_SWIGLU) {
+        constexpr int HALF = BN / 2;
+        __nv_bfloat16* H = static_cast<__nv_bfloat16*>(ep.out);
+#pragma unroll 1
+        for (int c = 0; c < HALF; c += 32) {
+          uint32_t g[32], u[32];
+          tmem_ld_32x32(taddr + c, g);
+          tmem_ld_32x32(taddr + HALF + c, u);
+          tmem_ld_wait();
+          const int64_t col0 = static_cast<int64_t>(n_blk) * HALF + c;
+          uint32_t packed[16];
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            const float g0 = __uint_as_float(g[i]), g1 = __uint_as_float(g[i + 1]);
+            const float s0 = __ldg(ep.scale + col0 + i), s1 = __ldg(ep.scale + col0 + i + 1);
+            const float h0 = __fdividef(g0, 1.0f + __expf(-g0)) * __uint_as_float(u[i]) * s0;
+            const float h1 = __fdividef(g1, 1.0f + __expf(-g1)) * __uint_as_float(u[i + 1]) * s1;
+            packed[i / 2] = pack_bf16(h0, h1);
+          }
+          if (row < ep.rows) {
+            uint4* dst = reinterpret_cast<uint4*>(H + row * ep.ld + col0);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t a[32];
+          tmem_ld_32x32(taddr + c, a);
+          tmem_ld_wait();
+          const int64_t col0 = static_cast<int64_t>(n_blk) * BN + c;
+          if (row < ep.rows) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+              const int64_t col = col0 + 4 * v;
+              if (col < ep.cols) {      // cols is a multiple of 4
+                float4 o = make_float4(__uint_as_float(a[4 * v]), __uint_as_float(a[4 * v + 1]),
+                                       __uint_as_float(a[4 * v + 2]), __uint_as_float(a[4 * v + 3]));
+                if (ep.R != nullptr) {
+                  const float4 r = *reinterpret_cast<const float4*>(ep.R + row * ep.ld + col);
+                  o.x += r.x; o.y += r.y; o.z += r.z; o.w += r.w;
+                }
+                if (ep.out_bf16) {
+                  uint2 pk = make_uint2(pack_bf16(o.x, o.y), pack_bf16(o.z, o.w));
+                  *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(ep.out) + row * ep.ld + col) = pk;
+                } else {
+                  *reinterpret_cast<float4*>(static_cast<float*>(ep.out) + row * ep.ld + col) = o;
+                }
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+  }
+
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(ep.status, kStatusTimeout);
+}
+
+constexpr int GU_BN = 256, GU_STAGES = 4;
+constexpr int DN_BN = 128, DN_STAGES = 6;
+
+}  // namespace
+
+cudaError_t tc_gemm_init() {
+  cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<GU_BN, GU_STAGES, EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       Cfg<GU_BN, GU_STAGES>::SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(tc_gemm_kernel<DN_BN, DN_STAGES, EPI_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Cfg<DN_BN, DN_STAGES>::SMEM_BYTES);
+}
+
+cudaError_t launch_tc_gateup(const TcGateUpArgs& a, int num_sms, cudaStream_t st) {
+  if (a.n == 0) return cudaSuccess;
+  const int m_blocks = static_cast<int>((a.n + BM - 1) / BM);
+  const int n_blocks = static_cast<int>(a.Ipad / (GU_BN / 2));
+  const int k_blocks = static_cast<int>((a.d + BK - 1) / BK);
+  EpiArgs ep{};
+  ep.scale = a.scale;
+  ep.out = a.H;
+  ep.rows = a.n;
+  ep.cols = a.Ipad;
+  ep.ld = a.Ipad;
+  ep.status = a.status;
+  const int tiles = m_blocks * n_blocks;
+  const int grid = tiles < num_sms ? tiles : num_sms;
+  tc_gemm_kernel<GU_BN, GU_STAGES, EPI_SWIGLU><<<grid, NUM_THREADS, Cfg<GU_BN, GU_STAGES>::SMEM_BYTES, st>>>(
+      a.tm_x, a.tm_w, ep, m_blocks, n_blocks, k_blocks);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_tc_down(const TcDownArgs& a, int num_sms, cudaStream_t st) {
+  if (a.n == 0) return cudaSuccess;
+  const int m_blocks = static_cast<int>((a.n + BM - 1) / BM);
+  const int n_blocks = static_cast<int>((a.d + DN_BN - 1) / DN_BN);
+  const int k_blocks = static_cast<int>(a.Ipad / BK);
+  EpiArgs ep{};
+  ep.R = a.R;
+  ep.out = a.Y;
+  ep.rows = a.n;
+  ep.cols = a.d;
+  ep.ld = a.d;
+  ep.out_bf16 = a.y_bf16;
+  ep.status = a.status;
+  const int tiles = m_blocks * n_blocks;
+  const int grid = tiles < num_sms ? tiles : num_sms;
+  tc_gemm_kernel<DN_BN, DN_STAGES, EPI_OUT><<<grid, NUM_THREADS, Cfg<DN_BN, DN_STAGES>::SMEM_BYTES, st>>>(
+      a.tm_h, a.tm_w, ep, m_blocks, n_blocks, k_blocks);
+  return cudaGetLastError();
+}
+
+}  // namespace mlpmoe

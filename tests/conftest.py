@@ -24,3 +24,12 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session")
+def lib():
+    """The Python binding over the C-ABI library, built in-tree if needed."""
+    from paper_2511_21089_b200 import build
+    build.build()
+    from paper_2511_21089_b200 import binding
+    return binding

@@ -1,0 +1,230 @@
+"""GPU parity of one MLPMoE layer against the oracle, through the C ABI: fp32 mode, the
+tensor-core prefill pair, the decode pair, Fade and pruning bookkeeping, edge cases."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_21089_b200 import synth
+from tests.helpers import TOL_BF16, TOL_FP32, Case, bits_of, dev_bf16, dev_f32, rel_err, stream_ptr
+
+pytestmark = pytest.mark.gpu
+
+
+def run_forward(lib, h, xd, n, d):
+    y = torch.empty((n, d), dtype=torch.float32, device="cuda")
+    lib.mlpmoe_forward(h, xd, y, n, stream_ptr())
+    torch.cuda.synchronize()
+    assert lib.mlpmoe_get_status(h) == lib.MLPMOE_OK
+    return y.cpu().numpy()
+
+
+def test_config1_fp32_equals_dense_swiglu(lib):
+    """Qwen2.5-0.5B MLP shape, fp32 weights, B = 8 x 608, 128 tokens, alpha = 1: the layer must
+    equal the dense SwiGLU MLP (Section 3.1)."""
+    c = Case((1, 0), 896, 4864, [608] * 8, bf16=False)
+    xh, xd = c.tokens((1, 0), 128)
+    h = c.create(lib, 128)
+    try:
+        y = run_forward(lib, h, xd, 128, 896)
+        ref = oracle.mlpmoe_forward(xh, *c.host, c.d_b)
+        dense = oracle.mlpmoe_forward(xh, *c.host, [4864])
+        assert rel_err(ref, dense) < 1e-12
+        assert rel_err(y, ref) <= TOL_FP32
+        b, segs = lib.mlpmoe_get_klist(h, 8, 4864)
+        assert b == list(range(8)) and segs == [(608 * i, 608) for i in range(8)]
+    finally:
+        lib.mlpmoe_destroy(h)
+
+
+@pytest.mark.parametrize("bf16", [True, False])
+@pytest.mark.parametrize("n", [65, 128, 200, 391])
+def test_small_layer_prefill(lib, bf16, n):
+    """Several tiles in every dimension and ragged tails: d = 320 (5 K-steps, 2.5 output tiles),
+    I = 400 -> padded to 512 (zero rows), unequal branches, non-unit alpha."""
+    d, I, d_b = 320, 400, [64, 160, 16, 160]
+    alpha = [1.0, 0.8, 1.2, -0.5]
+    c = Case((100, n), d, I, d_b, bf16=bf16, std=0.05, alpha=alpha)
+    xh, xd = c.tokens((100, n), n)
+    h = c.create(lib, 512)
+    try:
+        y = run_forward(lib, h, xd, n, d)
+        ref = oracle.mlpmoe_forward(xh, *c.host, d_b, c.alpha)
+        assert rel_err(y, ref) <= (TOL_BF16 if bf16 else TOL_FP32)
+    finally:
+        lib.mlpmoe_destroy(h)
+
+
+@pytest.mark.parametrize("n", [1, 2, 8, 16, 17, 32, 33, 64])
+def test_small_layer_decode(lib, n):
+    d, I, d_b = 320, 400, [64, 160, 16, 160]
+    c = Case((101, n), d, I, d_b, bf16=True, std=0.05, alpha=[1.0, 0.8, 1.2, -0.5])
+    xh, xd = c.tokens((101, n), n)
+    h = c.create(lib, 64)
+    try:
+        ref = oracle.mlpmoe_forward(xh, *c.host, d_b, c.alpha)
+        for _ in range(2):          # second call: the split-K arrival counters must have been reset
+            y = run_forward(lib, h, xd, n, d)
+            assert rel_err(y, ref) <= TOL_BF16
+    finally:
+        lib.mlpmoe_destroy(h)
+
+
+def test_layouts_agree(lib):
+    c = Case((102, 0), 128, 256, [128, 128], bf16=True, std=0.05)
+    xh, xd = c.tokens((102, 0), 100)
+    h0 = c.create(lib, 128, layout=lib.MLPMOE_LAYOUT_PAPER)
+    h1 = c.create(lib, 128, layout=lib.MLPMOE_LAYOUT_LINEAR)
+    try:
+        assert np.array_equal(run_forward(lib, h0, xd, 100, 128), run_forward(lib, h1, xd, 100, 128))
+    finally:
+        lib.mlpmoe_destroy(h0)
+        lib.mlpmoe_destroy(h1)
+
+
+@pytest.mark.parametrize("bf16", [True, False])
+def test_fade_masks_bit_exact(lib, bf16):
+    """Fractal Fade (Section 3.2): masked weights, non-zero counts and the forward after Fade."""
+    d, I, d_b = 128, 512, [64, 192, 128, 128]
+    c = Case((103, int(bf16)), d, I, d_b, bf16=bf16, std=0.02, alpha=[1.0, 0.9, 1.1, 1.05])
+    xh, xd = c.tokens((103, 1), 150)
+    h = c.create(lib, 256)
+    try:
+        lib.mlpmoe_fade(h, None, stream_ptr())
+        Fg, Fu = oracle.fade(c.host[0], c.host[1], d_b)
+        wg = torch.empty_like(c.dev[0]); wu = torch.empty_like(c.dev[1]); wd = torch.empty_like(c.dev[2])
+        lib.mlpmoe_get_weights(h, wg, wu, wd, stream_ptr())
+        torch.cuda.synchronize()
+        got = [synth.bf16_bits_to_f32(bits_of(w)) if bf16 else w.cpu().numpy() for w in (wg, wu, wd)]
+        assert np.array_equal(got[0], Fg) and np.array_equal(got[1], Fu) and np.array_equal(got[2], c.host[2])
+        assert lib.mlpmoe_nnz(h, 4) == oracle.nnz_per_branch(Fg, Fu, c.host[2], d_b)
+        y = run_forward(lib, h, xd, 150, d)
+        ref = oracle.mlpmoe_forward(xh, Fg, Fu, c.host[2], d_b, c.alpha)
+        assert rel_err(y, ref) <= (TOL_BF16 if bf16 else TOL_FP32)
+        # idempotent, and a custom schedule composes with it
+        lib.mlpmoe_fade(h, None, stream_ptr())
+        lib.mlpmoe_get_weights(h, wg, wu, None, stream_ptr())
+        torch.cuda.synchronize()
+        again = synth.bf16_bits_to_f32(bits_of(wg)) if bf16 else wg.cpu().numpy()
+        assert np.array_equal(again, Fg)
+        s = [0.5, 0.0, 0.25, 0.875]
+        lib.mlpmoe_fade(h, s, stream_ptr())
+        Fg2, Fu2 = oracle.fade(Fg, Fu, d_b, s)
+        lib.mlpmoe_get_weights(h, wg, wu, None, stream_ptr())
+        torch.cuda.synchronize()
+        got_g = synth.bf16_bits_to_f32(bits_of(wg)) if bf16 else wg.cpu().numpy()
+        got_u = synth.bf16_bits_to_f32(bits_of(wu)) if bf16 else wu.cpu().numpy()
+        assert np.array_equal(got_g, Fg2) and np.array_equal(got_u, Fu2)
+        with pytest.raises(lib.MlpmoeError) as e:
+            lib.mlpmoe_fade(h, [0.0, 1.0, 0.1, 0.1], stream_ptr())
+        assert e.value.status == lib.MLPMOE_ERR_BAD_SCHEDULE
+    finally:
+        lib.mlpmoe_destroy(h)
+
+
+@pytest.mark.parametrize("bf16", [True, False])
+def test_prune_schedule_bit_exact_and_forward(lib, bf16):
+    """Compensated Pruning (Section 3.3): effective gates, K-list and the forward."""
+    d, I, B = 128, 640, 8
+    d_b = [64, 128, 64, 64, 128, 64, 64, 64]
+    alpha = synth.uniform_f64((104, 0, 0, synth.T_ALPHA), B, 0.8, 1.2).astype(np.float32)
+    c = Case((104, int(bf16)), d, I, d_b, bf16=bf16, std=0.05, alpha=alpha)
+    xh, xd = c.tokens((104, 1), 130)
+    h = c.create(lib, 256)
+    try:
+        for keep, comp in ((synth.keep_set((104, 1), B, 2), True), (oracle.first_k_keep(B, 5), True),
+                           (synth.keep_set((104, 2), B, 7), False), ([True] * B, True)):
+            lib.mlpmoe_prune(h, keep, comp, stream_ptr())
+            a_ref = oracle.prune_alpha(c.alpha, keep, comp)
+            a_got = lib.mlpmoe_get_alpha(h, B)
+            assert np.array_equal(a_got.view(np.uint32), np.array(a_ref).astype(np.float32).view(np.uint32))
+            ref_b, ref_s = oracle.surviving_set(a_ref, *c.host, d_b)
+            assert lib.mlpmoe_get_klist(h, B, I) == (ref_b, ref_s)
+            assert lib.mlpmoe_get_active_neurons(h) == sum(l for _, l in ref_s)
+            y = run_forward(lib, h, xd, 130, d)
+            ref = oracle.mlpmoe_forward(xh, *c.host, d_b, a_ref)
+            assert rel_err(y, ref) <= (TOL_BF16 if bf16 else TOL_FP32)
+        lib.mlpmoe_prune_first_k(h, 3, stream_ptr())
+        assert np.array_equal(lib.mlpmoe_get_alpha(h, B)[:3],
+                              (np.float64(math.sqrt(8 / 3)) * alpha[:3].astype(np.float64)).astype(np.float32))
+        before = lib.mlpmoe_get_alpha(h, B)
+        with pytest.raises(lib.MlpmoeError) as e:
+            lib.mlpmoe_prune(h, [False] * B, True, stream_ptr())
+        assert e.value.status == lib.MLPMOE_ERR_EMPTY_KEEP_SET
+        assert np.array_equal(before, lib.mlpmoe_get_alpha(h, B))      # no state change on error
+    finally:
+        lib.mlpmoe_destroy(h)
+
+
+def test_dead_neurons_are_dropped(lib):
+    """Zero gate columns / up columns / down rows leave the schedule (single-neuron granularity)."""
+    d, I, d_b = 64, 256, [64, 64, 64, 64]
+    c = Case((105, 0), d, I, d_b, bf16=True, std=0.05)
+    for w in (c.bits, c.host):
+        w[0][:, 3] = 0
+        w[1][:, 70:75] = 0
+        w[2][130, :] = 0
+        w[0][:, 192:256] = 0          # a whole branch dies
+    c.dev = [dev_bf16(b) for b in c.bits]
+    xh, xd = c.tokens((105, 1), 90)
+    h = c.create(lib, 128)
+    try:
+        ref_b, ref_s = oracle.surviving_set([1.0] * 4, *c.host, d_b)
+        assert ref_b == [0, 1, 2]
+        assert lib.mlpmoe_get_klist(h, 4, I) == (ref_b, ref_s)
+        y = run_forward(lib, h, xd, 90, d)
+        assert rel_err(y, oracle.mlpmoe_forward(xh, *c.host, d_b)) <= TOL_BF16
+        xh1, xd1 = c.tokens((105, 2), 5)
+        y1 = run_forward(lib, h, xd1, 5, d)
+        assert rel_err(y1, oracle.mlpmoe_forward(xh1, *c.host, d_b)) <= TOL_BF16
+    finally:
+        lib.mlpmoe_destroy(h)
+
+
+def test_forward_ex_residual_bf16_out_and_argument_errors(lib):
+    d, I, d_b = 128, 256, [128, 128]
+    c = Case((106, 0), d, I, d_b, bf16=True, std=0.05)
+    h = c.create(lib, 256)
+    try:
+        for n in (7, 140):
+            xh, xd = c.tokens((106, n), n)
+            ref = oracle.mlpmoe_forward(xh, *c.host, d_b)
+            r = synth.normal_f32((106, n, 9), (n, d), 1.0)
+            rd = dev_f32(r)
+            y = torch.empty((n, d), dtype=torch.float32, device="cuda")
+            lib.mlpmoe_forward_ex(h, xd, y, n, rd, lib.MLPMOE_FP32, stream_ptr())
+            torch.cuda.synchronize()
+            assert rel_err(y.cpu().numpy() - r.astype(np.float64), ref) <= TOL_BF16
+            lib.mlpmoe_forward_ex(h, xd, rd, n, rd, lib.MLPMOE_FP32, stream_ptr())      # in place
+            torch.cuda.synchronize()
+            assert np.array_equal(rd.cpu().numpy(), y.cpu().numpy())
+            yb = torch.empty((n, d), dtype=torch.bfloat16, device="cuda")
+            lib.mlpmoe_forward_ex(h, xd, yb, n, None, lib.MLPMOE_BF16, stream_ptr())
+            torch.cuda.synchronize()
+            # bf16 output adds one rounding of y itself: 2^-9 relative per element
+            yb64 = yb.float().cpu().numpy().astype(np.float64)
+            assert np.max(np.abs(yb64 - ref) - np.abs(ref) * 2.0 ** -8) <= TOL_BF16 * np.sqrt(np.mean(ref ** 2))
+            # host-buffer entry point gives the same numbers as the device one
+            y0 = torch.empty((n, d), dtype=torch.float32, device="cuda")
+            lib.mlpmoe_forward(h, xd, y0, n, stream_ptr())
+            torch.cuda.synchronize()
+            xhost = xd.cpu().contiguous()
+            yhost = torch.empty((n, d), dtype=torch.float32)
+            lib.mlpmoe_forward_host(h, xhost, yhost, n, stream_ptr())
+            assert np.array_equal(yhost.numpy(), y0.cpu().numpy())
+        xh, xd = c.tokens((106, 1), 8)
+        y = torch.empty((8, d), dtype=torch.float32, device="cuda")
+        lib.mlpmoe_forward(h, xd, y, 0, stream_ptr())                   # n = 0: no-op
+        with pytest.raises(lib.MlpmoeError) as e:
+            lib.mlpmoe_forward(h, xd, y, 257, stream_ptr())             # > max_tokens
+        assert e.value.status == lib.MLPMOE_ERR_INVALID_ARG
+        with pytest.raises(lib.MlpmoeError):
+            lib.mlpmoe_forward(h, xd.data_ptr() + 2, y, 4, stream_ptr())   # misaligned x
+        with pytest.raises(lib.MlpmoeError):
+            lib.mlpmoe_forward(h, None, y, 4, stream_ptr())
+        assert lib.mlpmoe_get_launch_count(h) > 0
+        assert lib.mlpmoe_get_status(h) == lib.MLPMOE_OK
+    finally:
+        lib.mlpmoe_destroy(h)

@@ -1,0 +1,138 @@
+"""CPU-side tests of the library: it loads, exports every declared symbol, validates its
+arguments before touching CUDA, and its integer scheduling logic (Fade positions, effective
+gates, K-list) agrees bit-for-bit with the oracle."""
+import math
+import os
+import re
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2511_21089_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    header = open(os.path.join(ROOT, "include", "mlpmoe.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(mlpmoe_[a-z0-9_]+)\s*\(", header))
+    assert len(declared) >= 20
+    for name in declared:
+        assert hasattr(lib.lib, name), name
+    assert declared == set(lib.SIGNATURES)
+    assert lib.mlpmoe_status_string(0) == "ok"
+    assert "keep" in lib.mlpmoe_status_string(lib.MLPMOE_ERR_EMPTY_KEEP_SET)
+
+
+def test_create_rejects_bad_arguments_before_any_cuda_call(lib):
+    import ctypes
+    out = ctypes.c_void_p()
+    fake = 0x1000  # never dereferenced: the checks below fail first
+
+    def create(d, I, d_b, wg=fake, dtype=0, layout=0, max_tokens=16):
+        arr = (ctypes.c_int64 * len(d_b))(*d_b)
+        return lib.lib.mlpmoe_create(ctypes.byref(out), d, I, len(d_b), arr, wg, fake, fake, None, dtype, layout, max_tokens, None)
+
+    assert create(64, 64, [32, 16]) == lib.MLPMOE_ERR_BAD_PARTITION          # does not sum to d_inter
+    assert create(64, 64, [40, 24]) == lib.MLPMOE_ERR_BAD_PARTITION          # not multiples of 16
+    assert create(64, 64, [64, 0]) == lib.MLPMOE_ERR_BAD_PARTITION
+    assert create(64, 64, [32, 32], wg=None) == lib.MLPMOE_ERR_INVALID_ARG
+    assert create(0, 64, [64]) == lib.MLPMOE_ERR_INVALID_ARG
+    assert create(64, 64, [64], max_tokens=0) == lib.MLPMOE_ERR_INVALID_ARG
+    assert create(64, 64, [64], dtype=7) == lib.MLPMOE_ERR_INVALID_ARG
+    assert create(60, 64, [64]) == lib.MLPMOE_ERR_UNSUPPORTED                # d_model not a multiple of 8
+    assert out.value is None
+    # NULL handles are rejected everywhere, never dereferenced
+    assert lib.lib.mlpmoe_forward(None, fake, fake, 1, None) == lib.MLPMOE_ERR_INVALID_ARG
+    assert lib.lib.mlpmoe_fade(None, None, None) == lib.MLPMOE_ERR_INVALID_ARG
+    assert lib.lib.mlpmoe_prune(None, None, 1, None) == lib.MLPMOE_ERR_INVALID_ARG
+    assert lib.lib.mlpmoe_get_status(None) == lib.MLPMOE_ERR_INVALID_ARG
+    lib.mlpmoe_destroy(None)
+
+
+def test_fade_position_matches_oracle(lib):
+    rng = np.random.default_rng(1)
+    cases = [(0.0, 10), (0.5, 2), (0.9 * 31 / 32, 4096 * 448), (0.3, 1), (1e-300, 1 << 40), (0.999999999999, 1 << 40)]
+    for _ in range(300):
+        cases.append((float(rng.uniform(0, 1)), int(rng.integers(1, 1 << 36))))
+    for k in range(1, 60):                      # products that land exactly on, or next to, an integer
+        cases.append((k / 64.0, 64 * 977 + 1))
+        cases.append((math.nextafter(k / 64.0, 0.0), 64 * 977 + 1))
+    for s, m in cases:
+        assert lib.mlpmoe_host_fade_position(s, m) == oracle.fade_position(s, m)[0], (s, m)
+    for B in (4, 16, 32, 128):
+        sched = oracle.fade_schedule(B)
+        for b in range(B):
+            for m in (896 * 304, 4096 * 448, 4096 * 64, 17):
+                assert lib.mlpmoe_host_fade_position_default(b, B, m) == oracle.fade_position(sched[b], m)[0]
+    import ctypes
+    lo = ctypes.c_int64()
+    assert lib.lib.mlpmoe_host_fade_position(1.0, 10, ctypes.byref(lo)) == lib.MLPMOE_ERR_BAD_SCHEDULE
+    assert lib.lib.mlpmoe_host_fade_position(-0.1, 10, ctypes.byref(lo)) == lib.MLPMOE_ERR_BAD_SCHEDULE
+    assert lib.lib.mlpmoe_host_fade_position(float("nan"), 10, ctypes.byref(lo)) == lib.MLPMOE_ERR_BAD_SCHEDULE
+
+
+def test_prune_alpha_matches_oracle_bitwise(lib):
+    rng = np.random.default_rng(2)
+    for B in (4, 16, 64, 128):
+        alpha = rng.uniform(0.8, 1.2, size=B).astype(np.float32)
+        for n_drop in (0, 1, B // 4, B - 1):
+            keep = synth.keep_set((5, B, n_drop), B, n_drop)
+            for comp in (True, False):
+                ours = lib.mlpmoe_host_prune_alpha(alpha.tolist(), keep, comp)
+                ref = np.array(oracle.prune_alpha(alpha.astype(np.float64), keep, comp)).astype(np.float32)
+                assert np.array_equal(ours.view(np.uint32), ref.view(np.uint32))
+    with pytest.raises(lib.MlpmoeError) as e:
+        lib.mlpmoe_host_prune_alpha([1.0, 1.0], [False, False])
+    assert e.value.status == lib.MLPMOE_ERR_EMPTY_KEEP_SET
+    # the paper's first-K rule, literally
+    ours = lib.mlpmoe_host_prune_alpha([1.0] * 16, oracle.first_k_keep(16, 12))
+    assert np.array_equal(ours[:12], np.full(12, np.float32(math.sqrt(16 / 12)))) and np.all(ours[12:] == 0)
+
+
+def test_schedule_matches_oracle(lib):
+    rng = np.random.default_rng(3)
+    for trial in range(40):
+        B = int(rng.integers(1, 9))
+        d_b = [int(16 * rng.integers(1, 5)) for _ in range(B)]
+        I = sum(d_b)
+        alpha = rng.uniform(0.5, 1.5, size=B)
+        alpha[rng.uniform(size=B) < 0.3] = 0.0
+        p_dead = [0.0, 0.05, 0.5, 1.0][trial % 4]
+        live = rng.uniform(size=I) >= p_dead
+        # weights whose zero pattern gives exactly this liveness, through the three possible causes
+        Wg, Wu, Wd = np.ones((2, I)), np.ones((2, I)), np.ones((I, 2))
+        for j in np.nonzero(~live)[0]:
+            (Wg[:, j], Wu[:, j], Wd[j, :])[int(rng.integers(0, 3))][...] = 0
+        ref_b, ref_s = oracle.surviving_set(alpha, Wg, Wu, Wd, d_b)
+        got_b, got_s, n_act = lib.mlpmoe_host_schedule(d_b, alpha.astype(np.float32).tolist(), live.tolist())
+        assert got_b == ref_b and got_s == ref_s
+        assert n_act == sum(l for _, l in ref_s)
+    b, s, n = lib.mlpmoe_host_schedule([16, 32], [1.0, 1.0])
+    assert (b, s, n) == ([0, 1], [(0, 16), (16, 32)], 48)
+
+
+def test_synth_generators():
+    import torch
+    a = synth.normal_f32((1, 2, 3, 4), (3, 1 << 20), 0.02, threads=1)
+    b = synth.normal_f32((1, 2, 3, 4), (3, 1 << 20), 0.02, threads=8)
+    assert np.array_equal(a, b)                                   # independent of the thread count
+    assert abs(float(a.std()) - 0.02) < 2e-4 and abs(float(a.mean())) < 1e-4
+    assert not np.array_equal(a, synth.normal_f32((1, 2, 3, 5), (3, 1 << 20), 0.02))
+    bits = synth.f32_to_bf16_bits(a[0, :4096])
+    ref = torch.from_numpy(a[0, :4096].copy()).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(bits, ref)
+    assert np.array_equal(synth.bf16_bits_to_f32(bits), torch.from_numpy(a[0, :4096].copy()).to(torch.bfloat16).float().numpy())
+    for B in (4, 8, 16, 32, 64, 128):
+        p = synth.random_partition((9, B), 14336, B, 64)
+        assert len(p) == B and sum(p) == 14336 and all(w > 0 and w % 64 == 0 for w in p)
+        assert p == synth.random_partition((9, B), 14336, B, 64)
+    assert len(set(synth.random_partition((9, 16), 14336, 16, 64))) > 1
+    assert synth.equal_partition(4864, 16) == [304] * 16
+    k = synth.keep_set((7,), 16, 4)
+    assert sum(k) == 12 and k == synth.keep_set((7,), 16, 4)
+    assert [synth.n_drop_for_ratio(B, r) for B in (4, 32, 128) for r in (0.0, 0.1, 0.2, 0.4)] == \
+        [0, 0, 1, 2, 0, 3, 6, 13, 0, 13, 26, 51]
