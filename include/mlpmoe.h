@@ -202,6 +202,18 @@ mlpmoe_status_t mlpmoe_get_status(mlpmoe_handle_t h);
 mlpmoe_status_t mlpmoe_get_launch_count(mlpmoe_handle_t h, int64_t* launches);
 const char* mlpmoe_status_string(mlpmoe_status_t s);
 
+/*
+ * Per-kernel device timing for benchmarks (not in the paper).  With timing enabled, forward
+ * calls on this handle record CUDA events on their stream around each kernel they launch;
+ * nothing else changes.  Enabling allocates a fixed pool of events (a set-up call); once the
+ * pool is used up further launches are simply not timed.
+ *   mlpmoe_get_timing synchronises the device and returns, since the last call, the summed
+ *   duration in milliseconds and the number of timed launches of: [0] the gate|up kernel,
+ *   [1] the down kernel, [2] RMSNorm (stack calls only).  Both arrays have length 3.
+ */
+mlpmoe_status_t mlpmoe_set_timing(mlpmoe_handle_t h, int32_t enable);
+mlpmoe_status_t mlpmoe_get_timing(mlpmoe_handle_t h, double* ms, int64_t* launches);
+
 /* ------------------------------------------------------------------------- *
  * Host-only helpers: the scheduler's integer logic without any CUDA call
  * ------------------------------------------------------------------------- */

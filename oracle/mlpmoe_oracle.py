@@ -66,9 +66,9 @@ def branch_forward(x, W_gate, W_up, W_down, lo: int, hi: int, alpha_b: float) ->
     (Section 3.1, branch equation).  The sub-matrices are the column slice
     [lo, hi) of W_gate / W_up and the row slice [lo, hi) of W_down."""
     x = np.asarray(x, dtype=np.float64)
-    Wg = np.asarray(W_gate, dtype=np.float64)[:, lo:hi]
-    Wu = np.asarray(W_up, dtype=np.float64)[:, lo:hi]
-    Wd = np.asarray(W_down, dtype=np.float64)[lo:hi, :]
+    Wg = np.asarray(W_gate)[:, lo:hi].astype(np.float64)
+    Wu = np.asarray(W_up)[:, lo:hi].astype(np.float64)
+    Wd = np.asarray(W_down)[lo:hi, :].astype(np.float64)
     g = x @ Wg
     u = x @ Wu
     h = silu(g) * u

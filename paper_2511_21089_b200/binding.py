@@ -55,6 +55,8 @@ SIGNATURES = {
     "mlpmoe_get_status": (c_int32, [c_void_p]),
     "mlpmoe_get_launch_count": (c_int32, [c_void_p, POINTER(c_int64)]),
     "mlpmoe_status_string": (c_char_p, [c_int32]),
+    "mlpmoe_set_timing": (c_int32, [c_void_p, c_int32]),
+    "mlpmoe_get_timing": (c_int32, [c_void_p, POINTER(c_double), POINTER(c_int64)]),
     "mlpmoe_host_fade_position": (c_int32, [c_double, c_int64, POINTER(c_int64)]),
     "mlpmoe_host_fade_position_default": (c_int32, [c_int32, c_int32, c_int64, POINTER(c_int64)]),
     "mlpmoe_host_prune_alpha": (c_int32, [c_int32, POINTER(c_float), POINTER(c_uint8), c_int32, POINTER(c_float)]),
@@ -210,6 +212,18 @@ def mlpmoe_get_launch_count(h: int) -> int:
     v = c_int64()
     _check(lib.mlpmoe_get_launch_count(h, ctypes.byref(v)), "mlpmoe_get_launch_count")
     return v.value
+
+
+def mlpmoe_set_timing(h: int, enable: bool) -> None:
+    _check(lib.mlpmoe_set_timing(h, 1 if enable else 0), "mlpmoe_set_timing")
+
+
+def mlpmoe_get_timing(h: int):
+    """Returns ([ms gate|up, ms down, ms rmsnorm], [launch counts]) since the last call."""
+    ms = (c_double * 3)()
+    cnt = (c_int64 * 3)()
+    _check(lib.mlpmoe_get_timing(h, ms, cnt), "mlpmoe_get_timing")
+    return list(ms), list(cnt)
 
 
 def mlpmoe_host_fade_position(s: float, m: int) -> int:

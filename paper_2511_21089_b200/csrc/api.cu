@@ -171,12 +171,32 @@ struct mlpmoe_layer_s {
   uint32_t* status = nullptr;
   int64_t launches = 0;
   CUtensorMap tm_wgu, tm_wdt;
+  // optional per-kernel event timing
+  bool timing = false;
+  std::vector<cudaEvent_t> events;
+  size_t events_used = 0;
+  struct Span { int kind; size_t a, b; };
+  std::vector<Span> spans;
 };
 
 namespace {
 
+constexpr size_t kEventPool = 2048;
+enum { SPAN_GATEUP = 0, SPAN_DOWN = 1, SPAN_RMSNORM = 2 };
+
+// Records an event on `st` and returns its index in the pool, or -1 when timing is off / the pool is used up.
+long rec_event(mlpmoe_layer_s* h, cudaStream_t st) {
+  if (!h->timing || h->events_used >= h->events.size()) return -1;
+  if (cudaEventRecord(h->events[h->events_used], st) != cudaSuccess) return -1;
+  return static_cast<long>(h->events_used++);
+}
+void add_span(mlpmoe_layer_s* h, int kind, long a, long b) {
+  if (a >= 0 && b >= 0) h->spans.push_back({kind, static_cast<size_t>(a), static_cast<size_t>(b)});
+}
+
 void free_layer(mlpmoe_layer_s* h) {
   if (!h) return;
+  for (cudaEvent_t e : h->events) cudaEventDestroy(e);
   cudaFree(h->Wg_c); cudaFree(h->Wu_c); cudaFree(h->Wd_c);
   cudaFree(h->Wgu); cudaFree(h->WdT);
   cudaFree(h->scale); cudaFree(h->src_row); cudaFree(h->row_nnz);
@@ -234,8 +254,13 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
   if (y_dtype != MLPMOE_FP32 && !(y_dtype == MLPMOE_BF16 && h->dtype == MLPMOE_BF16)) return MLPMOE_ERR_UNSUPPORTED;
   if (h->dtype == MLPMOE_FP32) {
     float* H = static_cast<float*>(h->ws->H);
+    const long e0 = rec_event(h, st);
     CK(launch_simt_gateup(static_cast<const float*>(x), static_cast<const float*>(h->Wgu), h->scale, H, n, h->d, h->Ipad, st));
+    const long e1 = rec_event(h, st);
     CK(launch_simt_down(H, static_cast<const float*>(h->WdT), residual, static_cast<float*>(y), n, h->d, h->Ipad, st));
+    const long e2 = rec_event(h, st);
+    add_span(h, SPAN_GATEUP, e0, e1);
+    add_span(h, SPAN_DOWN, e1, e2);
     h->launches += 2;
     return MLPMOE_OK;
   }
@@ -261,7 +286,13 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
     if (splits < 1) splits = 1;
     a.splits = splits;
     a.status = h->status;
-    CK(launch_decode(a, h->num_sms, st));
+    const long e0 = rec_event(h, st);
+    CK(launch_decode_gateup(a, h->num_sms, st));
+    const long e1 = rec_event(h, st);
+    CK(launch_decode_down(a, h->num_sms, st));
+    const long e2 = rec_event(h, st);
+    add_span(h, SPAN_GATEUP, e0, e1);
+    add_span(h, SPAN_DOWN, e1, e2);
     h->launches += 2;
     return MLPMOE_OK;
   }
@@ -272,7 +303,9 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
   g.H = h->ws->H;
   g.n = n; g.d = h->d; g.Ipad = h->Ipad;
   g.status = h->status;
+  const long e0 = rec_event(h, st);
   CK(launch_tc_gateup(g, h->num_sms, st));
+  const long e1 = rec_event(h, st);
   TcDownArgs dn;
   if (!make_tmap(&dn.tm_h, h->ws->H, h->Ipad, n, h->Ipad, 128)) return MLPMOE_ERR_CUDA;
   dn.tm_w = h->tm_wdt;
@@ -282,6 +315,9 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
   dn.n = n; dn.d = h->d; dn.Ipad = h->Ipad;
   dn.status = h->status;
   CK(launch_tc_down(dn, h->num_sms, st));
+  const long e2 = rec_event(h, st);
+  add_span(h, SPAN_GATEUP, e0, e1);
+  add_span(h, SPAN_DOWN, e1, e2);
   h->launches += 2;
   return MLPMOE_OK;
 }
@@ -496,7 +532,10 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   for (int l = 0; l < n_layers; ++l) {
     mlpmoe_layer_s* h = layers[l];
+    const long e0 = rec_event(h, st);
     CK(launch_rmsnorm(x, h->ws->xnorm, n, h->d, eps, h->elem_size, st));
+    const long e1 = rec_event(h, st);
+    add_span(h, SPAN_RMSNORM, e0, e1);
     h->launches += 1;
     rc = forward_impl(h, h->ws->xnorm, x, n, x, MLPMOE_FP32, st);
     if (rc != MLPMOE_OK) return rc;
@@ -581,6 +620,35 @@ mlpmoe_status_t mlpmoe_get_status(mlpmoe_handle_t h) {
 mlpmoe_status_t mlpmoe_get_launch_count(mlpmoe_handle_t h, int64_t* launches) {
   if (!h || !launches) return MLPMOE_ERR_INVALID_ARG;
   *launches = h->launches;
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_set_timing(mlpmoe_handle_t h, int32_t enable) {
+  if (!h) return MLPMOE_ERR_INVALID_ARG;
+  if (enable && h->events.empty()) {
+    h->events.reserve(kEventPool);
+    for (size_t i = 0; i < kEventPool; ++i) {
+      cudaEvent_t e;
+      CK(cudaEventCreate(&e));
+      h->events.push_back(e);
+    }
+  }
+  h->timing = enable != 0;
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_get_timing(mlpmoe_handle_t h, double* ms, int64_t* launches) {
+  if (!h || !ms || !launches) return MLPMOE_ERR_INVALID_ARG;
+  CK(cudaDeviceSynchronize());
+  for (int k = 0; k < 3; ++k) { ms[k] = 0.0; launches[k] = 0; }
+  for (const auto& sp : h->spans) {
+    float t = 0.f;
+    CK(cudaEventElapsedTime(&t, h->events[sp.a], h->events[sp.b]));
+    ms[sp.kind] += t;
+    launches[sp.kind] += 1;
+  }
+  h->spans.clear();
+  h->events_used = 0;
   return MLPMOE_OK;
 }
 

@@ -335,15 +335,18 @@ cudaError_t decode_init() {
   return cudaFuncSetAttribute(decode_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_SMEM_BYTES);
 }
 
-cudaError_t launch_decode(const DecodeArgs& a, int num_sms, cudaStream_t st) {
+cudaError_t launch_decode_gateup(const DecodeArgs& a, int num_sms, cudaStream_t st) {
   if (a.n == 0) return cudaSuccess;
   const int tiles1 = static_cast<int>(a.Ipad / 128);
   const int kb1 = static_cast<int>((a.d + BK - 1) / BK);
   const int grid1 = tiles1 < num_sms ? tiles1 : num_sms;
   decode_gateup_kernel<<<grid1, NUM_THREADS, K1_SMEM_BYTES, st>>>(a.tm_w, a.tm_x, a.scale, static_cast<__nv_bfloat16*>(a.Hd),
                                                                  a.n, a.Ipad, tiles1, kb1, a.npad, a.status);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode_down(const DecodeArgs& a, int num_sms, cudaStream_t st) {
+  if (a.n == 0) return cudaSuccess;
   const int m_blocks = static_cast<int>((a.d + 127) / 128);
   const int items = m_blocks * a.splits;
   const int grid2 = items < num_sms ? items : num_sms;

@@ -87,7 +87,8 @@ struct DecodeArgs {
   int npad, splits;
   uint32_t* status;
 };
-cudaError_t launch_decode(const DecodeArgs& a, int num_sms, cudaStream_t st);
+cudaError_t launch_decode_gateup(const DecodeArgs& a, int num_sms, cudaStream_t st);
+cudaError_t launch_decode_down(const DecodeArgs& a, int num_sms, cudaStream_t st);
 cudaError_t decode_init();
 
 }  // namespace mlpmoe
