@@ -38,9 +38,9 @@ WORKLOAD = ("configs[1]: 24-layer MLP-only stack, Qwen2.5-0.5B shapes (d_model=8
             "RMSNorm + residual, 4096 tokens")
 
 
-def workload():
+def workload(layers=None):
     c = synth.CONFIGS[CFG]
-    return dict(d=c["d_model"], I=c["d_inter"], B=c["B"], n=c["n"], L=c["layers"], n_drop=c["n_drop"])
+    return dict(d=c["d_model"], I=c["d_inter"], B=c["B"], n=c["n"], L=layers or c["layers"], n_drop=c["n_drop"])
 
 
 def layer_inputs(layer: int, w):
@@ -101,7 +101,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    w = workload()
+    w = workload(args.layers)
     rows = 256
     tps, dt = time_oracle(w, rows, args.steps, args.warmup)
     cores = blas_threads()
@@ -180,7 +180,7 @@ def run_ours(args):
         dist.barrier()
     from paper_2511_21089_b200 import binding as lib
 
-    w = workload()
+    w = workload(args.layers)
     n, d, L = w["n"], w["d"], w["L"]
     stream = torch.cuda.current_stream()
     st = stream.cuda_stream
@@ -216,16 +216,25 @@ def run_ours(args):
     barrier()
     launches0 = sum(lib.mlpmoe_get_launch_count(h) for h in layers)
     for h in layers:
-        lib.mlpmoe_set_timing(h, bool(args.kernel_events))
+        lib.mlpmoe_set_timing(h, bool(args.kernel_events))     # allocates the event pools (set-up)
         lib.mlpmoe_get_timing(h)
+        lib.mlpmoe_set_timing(h, False)
     gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
     sampler = ClockSampler(gpu_id)
     time.sleep(0.3)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record(stream)
-    for _ in range(args.steps):
+    for i in range(args.steps):
+        # per-kernel events on every 8th step only: each record costs about a microsecond of stream time
+        timed = bool(args.kernel_events) and i % 8 == 0
+        if timed:
+            for h in layers:
+                lib.mlpmoe_set_timing(h, True)
         step()
+        if timed:
+            for h in layers:
+                lib.mlpmoe_set_timing(h, False)
     e1.record(stream)
     barrier()
     ms_total = e0.elapsed_time(e1)
@@ -267,7 +276,7 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
-            "config": {"workload": WORKLOAD, "l2": "inputs larger than L2: each step streams 0.47 GB of distinct weights",
+            "config": {"workload": WORKLOAD if L == synth.CONFIGS[CFG]["layers"] else WORKLOAD + f" [REDUCED to {L} layers]", "l2": "inputs larger than L2: each step streams 0.47 GB of distinct weights",
                        "surviving_neurons_per_layer": int(np.mean(active)), "tokens_per_rank": n},
             "clocks": clocks,
             "e2e": {"value": world * n / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": n * d * 4,
@@ -307,8 +316,9 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--layers", type=int, default=None, help="fewer layers of the same stack (profiling captures only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kernel-events", type=int, default=1, help="record per-kernel CUDA events in the timed region")
     ap.add_argument("--no-cpu-baseline", action="store_true")
