@@ -170,7 +170,8 @@ struct mlpmoe_layer_s {
   int max_splits = 1;
   uint32_t* status = nullptr;
   int64_t launches = 0;
-  CUtensorMap tm_wgu, tm_wdt;
+  CUtensorMap tm_wgu, tm_wdt;      // single-CTA boxes: 64 x 256 and 64 x 128
+  CUtensorMap tm_wgu_pair;         // CTA-pair box: 64 x 128
   // optional per-kernel event timing
   bool timing = false;
   std::vector<cudaEvent_t> events;
@@ -239,6 +240,7 @@ mlpmoe_status_t reschedule(mlpmoe_layer_s* h, cudaStream_t st) {
   if (h->dtype == MLPMOE_BF16) {
     if (!make_tmap(&h->tm_wgu, h->Wgu, h->d, 2 * h->Ipad, h->d, 256)) return MLPMOE_ERR_CUDA;
     if (!make_tmap(&h->tm_wdt, h->WdT, h->Ipad, h->d, h->Ipad, 128)) return MLPMOE_ERR_CUDA;
+    if (!make_tmap(&h->tm_wgu_pair, h->Wgu, h->d, 2 * h->Ipad, h->d, 128)) return MLPMOE_ERR_CUDA;
   }
   return MLPMOE_OK;
 }
@@ -296,25 +298,33 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
     h->launches += 2;
     return MLPMOE_OK;
   }
+  // n > 128: CTA pairs (256-token tiles); 65..128 tokens: one CTA per tile
+  const bool pair = n > 128;
   TcGateUpArgs g;
   if (!make_tmap(&g.tm_x, x, h->d, n, h->d, 128)) return MLPMOE_ERR_CUDA;
-  g.tm_w = h->tm_wgu;
+  g.tm_w = pair ? h->tm_wgu_pair : h->tm_wgu;
   g.scale = h->scale;
   g.H = h->ws->H;
   g.n = n; g.d = h->d; g.Ipad = h->Ipad;
   g.status = h->status;
-  const long e0 = rec_event(h, st);
-  CK(launch_tc_gateup(g, h->num_sms, st));
-  const long e1 = rec_event(h, st);
   TcDownArgs dn;
   if (!make_tmap(&dn.tm_h, h->ws->H, h->Ipad, n, h->Ipad, 128)) return MLPMOE_ERR_CUDA;
-  dn.tm_w = h->tm_wdt;
+  int bn = 128;
+  if (pair) {
+    bn = tc_pair_down_bn(n, h->d, h->num_sms);
+    if (!make_tmap(&dn.tm_w, h->WdT, h->Ipad, h->d, h->Ipad, bn / 2)) return MLPMOE_ERR_CUDA;
+  } else {
+    dn.tm_w = h->tm_wdt;
+  }
   dn.R = residual;
   dn.Y = y;
   dn.y_bf16 = y_dtype == MLPMOE_BF16;
   dn.n = n; dn.d = h->d; dn.Ipad = h->Ipad;
   dn.status = h->status;
-  CK(launch_tc_down(dn, h->num_sms, st));
+  const long e0 = rec_event(h, st);
+  CK(pair ? launch_tc_pair_gateup(g, h->num_sms, st) : launch_tc_gateup(g, h->num_sms, st));
+  const long e1 = rec_event(h, st);
+  CK(pair ? launch_tc_pair_down(dn, bn, h->num_sms, st) : launch_tc_down(dn, h->num_sms, st));
   const long e2 = rec_event(h, st);
   add_span(h, SPAN_GATEUP, e0, e1);
   add_span(h, SPAN_DOWN, e1, e2);
@@ -356,6 +366,7 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
   CK(cudaGetDeviceProperties(&prop, dev));
   if (prop.major != 10) return MLPMOE_ERR_UNSUPPORTED;     // kernels are built for sm_100a only
   CK(tc_gemm_init());
+  CK(tc_pair_init());
   CK(decode_init());
 
   mlpmoe_layer_s* h = new (std::nothrow) mlpmoe_layer_s();

@@ -70,6 +70,14 @@ cudaError_t launch_tc_gateup(const TcGateUpArgs& a, int num_sms, cudaStream_t st
 cudaError_t launch_tc_down(const TcDownArgs& a, int num_sms, cudaStream_t st);
 cudaError_t tc_gemm_init();   // opt in to the large dynamic shared memory sizes (once per process)
 
+// -------------------------------------------------------------- tc_gemm2.cu --
+// CTA-pair (cta_group::2) versions: tm_w of the gate|up call has box 64 x 128, tm_w of the down
+// call has box 64 x bn/2 (each CTA of a pair stages half of the weight rows of a tile).
+cudaError_t tc_pair_init();
+int tc_pair_down_bn(int64_t n, int64_t d, int num_sms);
+cudaError_t launch_tc_pair_gateup(const TcGateUpArgs& a, int num_sms, cudaStream_t st);
+cudaError_t launch_tc_pair_down(const TcDownArgs& a, int bn, int num_sms, cudaStream_t st);
+
 // ---------------------------------------------------------------- decode.cu --
 struct DecodeArgs {
   CUtensorMap tm_w;     // Wgu [2*Ipad x d]  box 64 x 64

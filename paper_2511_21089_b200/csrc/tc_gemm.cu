@@ -11,22 +11,13 @@
 //
 // Warp roles (192 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM owner + MMA issuer
 // (one lane), warps 2..5 = epilogue (TMEM lane quadrant = warp index mod 4).
-#include <cuda_bf16.h>
-
-#include "internal.h"
-#include "ptx.cuh"
+#include "tc_common.cuh"
 
 namespace mlpmoe {
 namespace {
 
 using namespace ptx;
-
-constexpr int BM = 128;        // rows of the A tile = UMMA M
-constexpr int BK = 64;         // K elements per stage: one 128-byte swizzled row of bf16
-constexpr int UMMA_K = 16;
-constexpr int NUM_THREADS = 192;
-
-enum { EPI_SWIGLU = 0, EPI_OUT = 1 };
+using namespace tc;
 
 template <int BN, int STAGES>
 struct Cfg {
@@ -37,22 +28,6 @@ struct Cfg {
   static constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;   // barriers + slack for 1024-byte alignment
   static constexpr int TMEM_COLS = 2 * BN;                      // two accumulator buffers
 };
-
-struct EpiArgs {
-  const float* scale;   // EPI_SWIGLU
-  const float* R;       // EPI_OUT, optional
-  void* out;            // H (bf16) or Y (fp32 / bf16)
-  int64_t rows;         // valid rows (tokens)
-  int64_t cols;         // valid output columns (EPI_OUT: d; EPI_SWIGLU: Ipad)
-  int64_t ld;           // output row pitch in elements
-  int out_bf16;         // EPI_OUT only
-  uint32_t* status;
-};
-
-__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
 
 template <int BN, int STAGES, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -111,6 +86,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
+      // tail: leave only after the MMAs have released every stage (their commits target these barriers)
+      for (int i = 0; ok && i < STAGES; ++i) {
+        if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag)) break;
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+      }
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
@@ -156,60 +136,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       tc_fence_after();
       const int64_t row = static_cast<int64_t>(m_blk) * BM + quad * 32 + lane;
       const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * BN) + (static_cast<uint32_t>(quad * 32) << 16);
-      if (EPI == EPI_SWIGLU) {
-        constexpr int HALF = BN / 2;
-        __nv_bfloat16* H = static_cast<__nv_bfloat16*>(ep.out);
-#pragma unroll 1
-        for (int c = 0; c < HALF; c += 32) {
-          uint32_t g[32], u[32];
-          tmem_ld_32x32(taddr + c, g);
-          tmem_ld_32x32(taddr + HALF + c, u);
-          tmem_ld_wait();
-          const int64_t col0 = static_cast<int64_t>(n_blk) * HALF + c;
-          uint32_t packed[16];
-#pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            const float g0 = __uint_as_float(g[i]), g1 = __uint_as_float(g[i + 1]);
-            const float s0 = __ldg(ep.scale + col0 + i), s1 = __ldg(ep.scale + col0 + i + 1);
-            const float h0 = __fdividef(g0, 1.0f + __expf(-g0)) * __uint_as_float(u[i]) * s0;
-            const float h1 = __fdividef(g1, 1.0f + __expf(-g1)) * __uint_as_float(u[i + 1]) * s1;
-            packed[i / 2] = pack_bf16(h0, h1);
-          }
-          if (row < ep.rows) {
-            uint4* dst = reinterpret_cast<uint4*>(H + row * ep.ld + col0);
-#pragma unroll
-            for (int v = 0; v < 4; ++v) dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-          }
-        }
-      } else {
-#pragma unroll 1
-        for (int c = 0; c < BN; c += 32) {
-          uint32_t a[32];
-          tmem_ld_32x32(taddr + c, a);
-          tmem_ld_wait();
-          const int64_t col0 = static_cast<int64_t>(n_blk) * BN + c;
-          if (row < ep.rows) {
-#pragma unroll
-            for (int v = 0; v < 8; ++v) {
-              const int64_t col = col0 + 4 * v;
-              if (col < ep.cols) {      // cols is a multiple of 4
-                float4 o = make_float4(__uint_as_float(a[4 * v]), __uint_as_float(a[4 * v + 1]),
-                                       __uint_as_float(a[4 * v + 2]), __uint_as_float(a[4 * v + 3]));
-                if (ep.R != nullptr) {
-                  const float4 r = *reinterpret_cast<const float4*>(ep.R + row * ep.ld + col);
-                  o.x += r.x; o.y += r.y; o.z += r.z; o.w += r.w;
-                }
-                if (ep.out_bf16) {
-                  uint2 pk = make_uint2(pack_bf16(o.x, o.y), pack_bf16(o.z, o.w));
-                  *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(ep.out) + row * ep.ld + col) = pk;
-                } else {
-                  *reinterpret_cast<float4*>(static_cast<float*>(ep.out) + row * ep.ld + col) = o;
-                }
-              }
-            }
-          }
-        }
-      }
+      if (EPI == EPI_SWIGLU)
+        epilogue_swiglu(taddr, ep, row, static_cast<int64_t>(n_blk) * (BN / 2), BN / 2);
+      else
+        epilogue_out(taddr, ep, row, static_cast<int64_t>(n_blk) * BN, BN);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tempty_bar[acc]);

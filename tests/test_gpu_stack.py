@@ -1,0 +1,109 @@
+"""GPU parity of the pre-norm residual stack x <- x + MLPMoE_l(RMSNorm(x)) against the oracle:
+a small stack compared element by element, and the full-size benchmark workload (24 layers,
+Qwen2.5-0.5B shapes, 4096 tokens, 12 of 16 branches kept) compared on sampled token rows."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_21089_b200 import synth
+from tests.helpers import TOL_BF16, TOL_FP32, Case, dev_bf16, dev_f32, rel_err, stream_ptr
+
+pytestmark = pytest.mark.gpu
+
+
+def test_rmsnorm_kernel(lib):
+    x = synth.normal_f32((200, 0), (300, 320), 3.0)
+    xd = dev_f32(x)
+    ref = oracle.rmsnorm(x)
+    r32 = torch.empty((300, 320), dtype=torch.float32, device="cuda")
+    lib.mlpmoe_rmsnorm(xd, r32, 300, 320, 1e-6, lib.MLPMOE_FP32, stream_ptr())
+    rb = torch.empty((300, 320), dtype=torch.bfloat16, device="cuda")
+    lib.mlpmoe_rmsnorm(xd, rb, 300, 320, 1e-6, lib.MLPMOE_BF16, stream_ptr())
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(r32.cpu().numpy(), ref, rtol=2e-6, atol=1e-7)
+    # bf16 output: the rounding of a value within 2e-6 of the exact one, i.e. at most one bf16 step away
+    got = rb.float().cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(got - oracle.round_to_bf16(ref)) / np.maximum(np.abs(ref), 1e-30)) <= 2.0 ** -7
+    assert np.mean(got != oracle.round_to_bf16(ref)) < 1e-3
+
+
+@pytest.mark.parametrize("bf16", [True, False])
+@pytest.mark.parametrize("n", [24, 300])
+def test_small_stack(lib, bf16, n):
+    d, I, d_b, L = 256, 384, [128, 64, 192], 3
+    cases, handles, layers = [], [], []
+    try:
+        for l in range(L):
+            c = Case((201, l, int(bf16)), d, I, d_b, bf16=bf16, std=0.05, alpha=[1.0, 0.9, 1.1])
+            h = c.create(lib, 512)
+            keep = [True, l != 1, True]
+            lib.mlpmoe_prune(h, keep, True, stream_ptr())
+            if handles:
+                lib.mlpmoe_share_workspace(h, handles[0])
+            handles.append(h)
+            layers.append((*c.host, d_b, oracle.prune_alpha(c.alpha, keep)))
+        x = synth.normal_f32((201, 9, n), (n, d), 1.0)
+        xd = dev_f32(x)
+        lib.mlpmoe_stack_forward(handles, xd, n, 1e-6, stream_ptr())
+        torch.cuda.synchronize()
+        ref = oracle.stack_forward(x, layers, bf16_activations=bf16)
+        assert rel_err(xd.cpu().numpy(), ref) <= (TOL_BF16 if bf16 else TOL_FP32)
+        # host-buffer entry point
+        yh = torch.empty((n, d), dtype=torch.float32)
+        lib.mlpmoe_stack_forward_host(handles, torch.from_numpy(x), yh, n, 1e-6, stream_ptr())
+        assert np.array_equal(yh.numpy(), xd.cpu().numpy())
+        assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
+    finally:
+        for h in handles[1:] + handles[:1]:
+            lib.mlpmoe_destroy(h)
+
+
+def test_config2_full_size_sampled_rows(lib):
+    """The benchmark's workload in the benchmark's launch configuration; the oracle runs the
+    sampled rows through all 24 layers (rows are independent)."""
+    cfg = synth.CONFIGS[2]
+    d, I, B, n, L = cfg["d_model"], cfg["d_inter"], cfg["B"], cfg["n"], cfg["layers"]
+    d_b = synth.equal_partition(I, B)
+    handles, layers = [], []
+    try:
+        for l in range(L):
+            bits = synth.layer_weights(2, l, d, I, 0.02, bf16=True)
+            keep = synth.keep_set((synth.BASE_SEED, 2, l, synth.T_KEEP), B, cfg["n_drop"])
+            dev = [dev_bf16(b) for b in bits]
+            h = lib.mlpmoe_create(d, I, d_b, dev[0], dev[1], dev[2], None, lib.MLPMOE_BF16, lib.MLPMOE_LAYOUT_PAPER, n, stream_ptr())
+            lib.mlpmoe_prune(h, keep, True, stream_ptr())
+            if handles:
+                lib.mlpmoe_share_workspace(h, handles[0])
+            handles.append(h)
+            alpha = oracle.prune_alpha([1.0] * B, keep)
+            host = [synth.bf16_bits_to_f32(b) for b in bits]
+            layers.append((*host, d_b, alpha))
+            # the schedule is bit-exact: kept branches, one full segment each
+            assert np.array_equal(lib.mlpmoe_get_alpha(h, B).view(np.uint32), np.array(alpha).astype(np.float32).view(np.uint32))
+            assert lib.mlpmoe_get_klist(h, B, I) == oracle.surviving_set(alpha, *host, d_b)
+            assert lib.mlpmoe_get_active_neurons(h) == 12 * 304
+        x = synth.tokens(2, n, d)
+        xd = dev_f32(x)
+        lib.mlpmoe_stack_forward(handles, xd, n, 1e-6, stream_ptr())
+        torch.cuda.synchronize()
+        rows = sorted(set([0, 1, 127, 128, 255, 256, 2047, 2048, n - 129, n - 1] +
+                          list(np.random.default_rng(5).integers(0, n, size=38))))
+        ref = oracle.stack_forward(x[rows], layers, bf16_activations=True)
+        got = xd.cpu().numpy()
+        assert np.isfinite(got).all()
+        assert rel_err(got[rows], ref) <= TOL_BF16
+        # the layer's own contribution (output minus input) at the last layer, fed the oracle's layer input
+        _, inputs = oracle.stack_forward(x[rows], layers, bf16_activations=True, return_layer_inputs=True)
+        xin = np.zeros((n, d), dtype=np.float32)
+        xin[:len(rows)] = inputs[-1].astype(np.float32)
+        xin_d = dev_f32(xin)
+        lib.mlpmoe_stack_forward(handles[-1:], xin_d, n, 1e-6, stream_ptr())
+        torch.cuda.synchronize()
+        delta_ref = ref - inputs[-1]
+        delta_got = xin_d.cpu().numpy()[:len(rows)].astype(np.float64) - xin[:len(rows)].astype(np.float64)
+        assert rel_err(delta_got, delta_ref) <= TOL_BF16
+        assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
+    finally:
+        for h in handles[1:] + handles[:1]:
+            lib.mlpmoe_destroy(h)
