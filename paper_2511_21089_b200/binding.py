@@ -15,7 +15,7 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmlpmoe_b200.so")
+LIB_PATH = os.environ.get("MLPMOE_LIB_PATH") or os.path.join(_HERE, "libmlpmoe_b200.so")
 
 MLPMOE_OK = 0
 MLPMOE_ERR_INVALID_ARG = 1
