@@ -55,17 +55,22 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// bf16 row-major matrix [outer x inner] with row pitch `pitch_elems`; box = 64 x box_outer, 128-byte swizzle.
-bool make_tmap(CUtensorMap* m, const void* ptr, int64_t inner, int64_t outer, int64_t pitch_elems, int box_outer) {
+// Row-major matrix [outer x inner] of bf16 (elem_size 2) or fp32 (4) with row pitch `pitch_elems`;
+// box = 128 bytes x box_outer rows, 128-byte swizzle.
+bool make_tmap_t(CUtensorMap* m, const void* ptr, int64_t inner, int64_t outer, int64_t pitch_elems, int box_outer,
+                 int elem_size) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {static_cast<cuuint64_t>(inner), static_cast<cuuint64_t>(outer)};
-  cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch_elems) * 2};
-  cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_outer)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch_elems) * elem_size};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / elem_size), static_cast<cuuint32_t>(box_outer)};
   cuuint32_t estr[2] = {1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return fn(m, elem_size == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+            const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+bool make_tmap(CUtensorMap* m, const void* ptr, int64_t inner, int64_t outer, int64_t pitch_elems, int box_outer) {
+  return make_tmap_t(m, ptr, inner, outer, pitch_elems, box_outer, 2);
 }
 
 // ------------------------------------------------------------ host logic ----
@@ -313,6 +318,12 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
   if (pair) {
     bn = tc_pair_down_bn(n, h->d, h->num_sms);
     if (!make_tmap(&dn.tm_w, h->WdT, h->Ipad, h->d, h->Ipad, bn / 2)) return MLPMOE_ERR_CUDA;
+    if (!make_tmap(&g.tm_out, h->ws->H, h->Ipad, n, h->Ipad, 32)) return MLPMOE_ERR_CUDA;
+    if (y_dtype == MLPMOE_FP32) {
+      if (!make_tmap_t(&dn.tm_out, y, h->d, n, h->d, 32, 4)) return MLPMOE_ERR_CUDA;
+    } else {
+      dn.tm_out = dn.tm_h;     // not used by the direct epilogue; any valid map
+    }
   } else {
     dn.tm_w = h->tm_wdt;
   }

@@ -52,6 +52,7 @@ cudaError_t launch_simt_down(const float* H, const float* WdT, const float* R, f
 struct TcGateUpArgs {
   CUtensorMap tm_x;     // X   [n x d]            bf16, box 64 x 128, 128B swizzle
   CUtensorMap tm_w;     // Wgu [2*Ipad x d]       bf16, box 64 x 256
+  CUtensorMap tm_out;   // H   [n x Ipad]         bf16, box 64 x 32 (CTA-pair kernel's TMA-store epilogue)
   const float* scale;   // [Ipad]
   void* H;              // [n x Ipad] bf16
   int64_t n, d, Ipad;
@@ -60,6 +61,7 @@ struct TcGateUpArgs {
 struct TcDownArgs {
   CUtensorMap tm_h;     // H   [n x Ipad]         bf16, box 64 x 128
   CUtensorMap tm_w;     // WdT [d x Ipad]         bf16, box 64 x 128
+  CUtensorMap tm_out;   // Y   [n x d]            fp32, box 32 x 32 (CTA-pair kernel's TMA-store epilogue)
   const float* R;       // optional fp32 residual [n x d]
   void* Y;              // [n x d] fp32 or bf16
   int y_bf16;

@@ -181,28 +181,24 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rn(float f) {
   return static_cast<uint16_t>(u >> 16);
 }
 
+// One warp per token row: pass 1 sums the squares, pass 2 re-reads the row (now in L1) and writes
+// the normalised values.  HBM traffic = one read of x and one write of r.
 template <bool OUT_BF16>
-__global__ void rmsnorm_kernel(const float* __restrict__ x, void* __restrict__ r, int64_t n, int64_t d, float eps) {
-  const int64_t t = blockIdx.x;
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ x, void* __restrict__ r, int64_t n, int64_t d,
+                                                      float eps) {
+  const int64_t t = static_cast<int64_t>(blockIdx.x) * (blockDim.x / 32) + threadIdx.x / 32;
+  const int lane = threadIdx.x % 32;
+  if (t >= n) return;
   const float4* row = reinterpret_cast<const float4*>(x + t * d);
   const int64_t nv = d / 4;
   float ss = 0.f;
-  for (int64_t v = threadIdx.x; v < nv; v += blockDim.x) {
+  for (int64_t v = lane; v < nv; v += 32) {
     const float4 a = row[v];
     ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
   }
-  __shared__ float red[32];
   for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
-  if (threadIdx.x % 32 == 0) red[threadIdx.x / 32] = ss;
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    float v = threadIdx.x < blockDim.x / 32 ? red[threadIdx.x] : 0.f;
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    if (threadIdx.x == 0) red[0] = v;
-  }
-  __syncthreads();
-  const float inv = 1.0f / sqrtf(red[0] / static_cast<float>(d) + eps);
-  for (int64_t v = threadIdx.x; v < nv; v += blockDim.x) {
+  const float inv = 1.0f / sqrtf(ss / static_cast<float>(d) + eps);
+  for (int64_t v = lane; v < nv; v += 32) {
     const float4 a = row[v];
     if (OUT_BF16) {
       uint2 o;
@@ -298,9 +294,9 @@ cudaError_t launch_fade(const FadeSeg* segs_host, int nseg, void* work, int elem
 cudaError_t launch_rmsnorm(const float* x, void* r, int64_t n, int64_t d, float eps, int out_elem_size, cudaStream_t st) {
   if (n == 0) return cudaSuccess;
   if (out_elem_size == 2)
-    rmsnorm_kernel<true><<<static_cast<unsigned>(n), 256, 0, st>>>(x, r, n, d, eps);
+    rmsnorm_kernel<true><<<cdiv(n, 8), 256, 0, st>>>(x, r, n, d, eps);
   else
-    rmsnorm_kernel<false><<<static_cast<unsigned>(n), 256, 0, st>>>(x, r, n, d, eps);
+    rmsnorm_kernel<false><<<cdiv(n, 8), 256, 0, st>>>(x, r, n, d, eps);
   return cudaGetLastError();
 }
 

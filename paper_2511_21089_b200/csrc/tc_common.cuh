@@ -98,5 +98,111 @@ __device__ __forceinline__ void epilogue_out(uint32_t taddr, const EpiArgs& ep, 
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Epilogues that leave through shared memory and TMA: each epilogue warp owns two 4 KB staging
+// tiles (32 rows x 128 bytes, 128-byte swizzle, 1024-byte aligned) and alternates between them.
+// Lane r writes row r; the 16-byte chunk c of a row sits at chunk position c ^ (r % 8), which is
+// both what the swizzled tensor map expects and free of bank conflicts.  One lane issues the
+// bulk tensor store, which is clipped to the tensor's extent (rows >= n, columns >= d).
+// ---------------------------------------------------------------------------------------------
+constexpr int STAGING_TILE_BYTES = 4096;
+constexpr int STAGING_BYTES_PER_WARP = 2 * STAGING_TILE_BYTES;
+
+__device__ __forceinline__ void staging_write16(uint8_t* tile, int lane, int chunk, uint4 v) {
+  *reinterpret_cast<uint4*>(tile + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = v;
+}
+
+__device__ __forceinline__ float silu_mul(uint32_t g_bits, uint32_t u_bits, float sc) {
+  const float g = __uint_as_float(g_bits);
+  return __fdividef(g, 1.0f + __expf(-g)) * __uint_as_float(u_bits) * sc;
+}
+
+// gate|up epilogue for one 128-neuron tile.  tm_h: bf16 [n x Ipad], box 64 x 32.  `tiles_stored`
+// counts this warp's staging tiles so far (selects the buffer).  `release` is called as soon as
+// the accumulator has been read completely, before the arithmetic and the stores finish.
+template <typename Release>
+__device__ __forceinline__ void epilogue_swiglu_tma(uint32_t taddr, const float* __restrict__ scale, const CUtensorMap* tm_h,
+                                                    uint8_t* staging, uint32_t& tiles_stored, int lane, int32_t row0,
+                                                    int32_t neuron0, Release release) {
+  uint32_t g[2][32], u[2][32];
+  ptx::tmem_ld_32x32(taddr, g[0]);
+  ptx::tmem_ld_32x32(taddr + 128, u[0]);
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {          // four groups of 32 neurons
+    ptx::tmem_ld_wait();
+    if (s < 3) {
+      ptx::tmem_ld_32x32(taddr + 32 * (s + 1), g[(s + 1) & 1]);
+      ptx::tmem_ld_32x32(taddr + 128 + 32 * (s + 1), u[(s + 1) & 1]);
+    } else {
+      release();
+    }
+    uint8_t* tile = staging + (tiles_stored & 1u) * STAGING_TILE_BYTES;
+    if ((s & 1) == 0) {                   // a new 64-neuron staging tile: its previous store must have been read
+      if (lane == 0) ptx::tma_store_wait_read<1>();
+      __syncwarp();
+    }
+    const float4* sc4 = reinterpret_cast<const float4*>(scale + neuron0 + 32 * s);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {         // 8 neurons -> one 16-byte chunk
+      const float4 s0 = __ldg(sc4 + 2 * q), s1 = __ldg(sc4 + 2 * q + 1);
+      const uint32_t* gg = &g[s & 1][8 * q];
+      const uint32_t* uu = &u[s & 1][8 * q];
+      uint4 v;
+      v.x = pack_bf16(silu_mul(gg[0], uu[0], s0.x), silu_mul(gg[1], uu[1], s0.y));
+      v.y = pack_bf16(silu_mul(gg[2], uu[2], s0.z), silu_mul(gg[3], uu[3], s0.w));
+      v.z = pack_bf16(silu_mul(gg[4], uu[4], s1.x), silu_mul(gg[5], uu[5], s1.y));
+      v.w = pack_bf16(silu_mul(gg[6], uu[6], s1.z), silu_mul(gg[7], uu[7], s1.w));
+      staging_write16(tile, lane, 4 * (s & 1) + q, v);
+    }
+    if ((s & 1) == 1) {
+      ptx::fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        ptx::tma_store_2d(tm_h, tile, neuron0 + 32 * (s - 1), row0);
+        ptx::tma_store_commit();
+      }
+      ++tiles_stored;
+    }
+  }
+}
+
+// down epilogue, fp32 output: bn accumulator columns (a multiple of 32) starting at col_base.
+// tm_y: fp32 [n x d], box 32 x 32.  accumulate != 0 adds onto Y (the residual stream updated
+// in place), otherwise Y is overwritten.
+template <typename Release>
+__device__ __forceinline__ void epilogue_out_tma(uint32_t taddr, const CUtensorMap* tm_y, uint8_t* staging,
+                                                 uint32_t& tiles_stored, int lane, int32_t row0, int32_t col_base, int bn,
+                                                 int accumulate, Release release) {
+  uint32_t a[2][32];
+  ptx::tmem_ld_32x32(taddr, a[0]);
+  const int chunks = bn / 32;
+#pragma unroll 1
+  for (int c = 0; c < chunks; c += 2) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int cc = c + e;
+      if (cc < chunks) {
+        ptx::tmem_ld_wait();
+        if (cc + 1 < chunks) ptx::tmem_ld_32x32(taddr + 32 * (cc + 1), a[(e + 1) & 1]);
+        else release();
+        uint8_t* tile = staging + (tiles_stored & 1u) * STAGING_TILE_BYTES;
+        if (lane == 0) ptx::tma_store_wait_read<1>();
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          staging_write16(tile, lane, q, make_uint4(a[e][4 * q], a[e][4 * q + 1], a[e][4 * q + 2], a[e][4 * q + 3]));
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          if (accumulate) ptx::tma_reduce_add_2d(tm_y, tile, col_base + 32 * cc, row0);
+          else ptx::tma_store_2d(tm_y, tile, col_base + 32 * cc, row0);
+          ptx::tma_store_commit();
+        }
+        ++tiles_stored;
+      }
+    }
+  }
+}
+
 }  // namespace tc
 }  // namespace mlpmoe

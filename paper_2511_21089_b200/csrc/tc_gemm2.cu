@@ -27,16 +27,20 @@ constexpr int STAGES = 6;
 constexpr int A_BYTES = BM * BK * 2;                 // 16 KB
 constexpr int B_HALF_MAX_BYTES = 128 * BK * 2;       // up to 128 weight rows per CTA
 constexpr int STAGE_BYTES = A_BYTES + B_HALF_MAX_BYTES;
-constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+constexpr int STAGING_OFFSET = STAGES * STAGE_BYTES;                 // epilogue staging tiles, 8 KB per epilogue warp
+constexpr int BAR_OFFSET = STAGING_OFFSET + 4 * STAGING_BYTES_PER_WARP;
 constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;
+static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 constexpr int ACC_STRIDE = 256;                      // TMEM columns per accumulator buffer
 constexpr int TMEM_COLS = 512;
 constexpr uint64_t WAIT_NS = 1000000000ull;
+enum { OUT_DIRECT = 0, OUT_TMA_STORE = 1, OUT_TMA_ADD = 2 };   // how the down epilogue leaves
 
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
-tc_pair_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const EpiArgs ep,
-                    int num_m_pairs, int num_n_blocks, int num_k_blocks, int bn) {
+tc_pair_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                    const __grid_constant__ CUtensorMap tm_out, const EpiArgs ep, int num_m_pairs, int num_n_blocks,
+                    int num_k_blocks, int bn, int out_mode) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + BAR_OFFSET);   // used in the even CTA
@@ -137,26 +141,37 @@ tc_pair_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   } else {
     // ---------------------------------------------------------------- epilogue
     const int quad = warp % 4;
+    uint8_t* staging = smem + STAGING_OFFSET + (warp - 2) * STAGING_BYTES_PER_WARP;
+    uint32_t tiles_stored = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
+    if (lane == 0) prefetch_tensormap(&tm_out);
     for (int tile = first_tile; tile < num_tiles; tile += tile_step) {
       const int m_pair = tile % num_m_pairs, n_blk = tile / num_m_pairs;
       bool ok = mbar_wait_bounded(&tfull_bar[acc], acc_phase, abort_flag, WAIT_NS);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int64_t row = static_cast<int64_t>(m_pair * 2 + static_cast<int>(rank)) * BM + quad * 32 + lane;
+      const int32_t row0 = (m_pair * 2 + static_cast<int>(rank)) * BM + quad * 32;
       const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * ACC_STRIDE) + (static_cast<uint32_t>(quad * 32) << 16);
-      if (EPI == EPI_SWIGLU)
-        epilogue_swiglu(taddr, ep, row, static_cast<int64_t>(n_blk) * 128, 128);
-      else
-        epilogue_out(taddr, ep, row, static_cast<int64_t>(n_blk) * BN, BN);
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty_bar[acc]), 0));
+      const uint32_t tempty_even = map_to_cta(smem_u32(&tempty_bar[acc]), 0);
+      auto release = [&]() {               // the accumulator buffer may be overwritten by the next tile's MMAs
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(tempty_even);
+      };
+      if (EPI == EPI_SWIGLU) {
+        epilogue_swiglu_tma(taddr, ep.scale, &tm_out, staging, tiles_stored, lane, row0, n_blk * 128, release);
+      } else if (out_mode != OUT_DIRECT) {
+        epilogue_out_tma(taddr, &tm_out, staging, tiles_stored, lane, row0, n_blk * BN, BN, out_mode == OUT_TMA_ADD, release);
+      } else {
+        epilogue_out(taddr, ep, static_cast<int64_t>(row0) + lane, static_cast<int64_t>(n_blk) * BN, BN);
+        release();
+      }
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
+    if (lane == 0) tma_store_wait_all<0>();   // this warp's bulk stores have completed
   }
 
   __syncwarp();
@@ -207,7 +222,8 @@ cudaError_t launch_tc_pair_gateup(const TcGateUpArgs& a, int num_sms, cudaStream
   ep.status = a.status;
   const int tiles = m_pairs * n_blocks;
   const int pairs = tiles < num_sms / 2 ? tiles : num_sms / 2;
-  tc_pair_gemm_kernel<EPI_SWIGLU><<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(a.tm_x, a.tm_w, ep, m_pairs, n_blocks, k_blocks, 256);
+  tc_pair_gemm_kernel<EPI_SWIGLU><<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(a.tm_x, a.tm_w, a.tm_out, ep, m_pairs, n_blocks,
+                                                                            k_blocks, 256, OUT_TMA_STORE);
   return cudaGetLastError();
 }
 
@@ -226,7 +242,13 @@ cudaError_t launch_tc_pair_down(const TcDownArgs& a, int bn, int num_sms, cudaSt
   ep.status = a.status;
   const int tiles = m_pairs * n_blocks;
   const int pairs = tiles < num_sms / 2 ? tiles : num_sms / 2;
-  tc_pair_gemm_kernel<EPI_OUT><<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(a.tm_h, a.tm_w, ep, m_pairs, n_blocks, k_blocks, bn);
+  // fp32 output leaves through TMA: plain store without a residual, add-in-place when the residual
+  // is the output buffer itself; other combinations use the direct (per-thread) epilogue
+  int mode = OUT_DIRECT;
+  if (!a.y_bf16 && a.R == nullptr) mode = OUT_TMA_STORE;
+  else if (!a.y_bf16 && a.R == a.Y) mode = OUT_TMA_ADD;
+  tc_pair_gemm_kernel<EPI_OUT><<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(a.tm_h, a.tm_w, a.tm_out, ep, m_pairs, n_blocks,
+                                                                         k_blocks, bn, mode);
   return cudaGetLastError();
 }
 
