@@ -85,6 +85,8 @@ decode_gateup_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_launch_dependents();          // the next kernel may begin its set-up
+  griddep_wait();                       // inputs written by earlier kernels are complete and visible
   const uint32_t stage_tx = K1_W_BYTES + static_cast<uint32_t>(npad) * BK * 2;
 
   if (warp == 0) {
@@ -197,6 +199,8 @@ decode_down_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_launch_dependents();          // the next kernel may begin its set-up
+  griddep_wait();                       // inputs written by earlier kernels are complete and visible
   const uint32_t stage_tx = K2_W_BYTES + static_cast<uint32_t>(npad) * BK * 2;
   const int num_items = num_m_blocks * splits;
 
@@ -340,9 +344,8 @@ cudaError_t launch_decode_gateup(const DecodeArgs& a, int num_sms, cudaStream_t 
   const int tiles1 = static_cast<int>(a.Ipad / 128);
   const int kb1 = static_cast<int>((a.d + BK - 1) / BK);
   const int grid1 = tiles1 < num_sms ? tiles1 : num_sms;
-  decode_gateup_kernel<<<grid1, NUM_THREADS, K1_SMEM_BYTES, st>>>(a.tm_w, a.tm_x, a.scale, static_cast<__nv_bfloat16*>(a.Hd),
-                                                                 a.n, a.Ipad, tiles1, kb1, a.npad, a.status);
-  return cudaGetLastError();
+  return launch_pdl(decode_gateup_kernel, dim3(grid1), dim3(NUM_THREADS), K1_SMEM_BYTES, st, a.tm_w, a.tm_x, a.scale,
+                    static_cast<__nv_bfloat16*>(a.Hd), a.n, a.Ipad, tiles1, kb1, a.npad, a.status);
 }
 
 cudaError_t launch_decode_down(const DecodeArgs& a, int num_sms, cudaStream_t st) {
@@ -350,10 +353,8 @@ cudaError_t launch_decode_down(const DecodeArgs& a, int num_sms, cudaStream_t st
   const int m_blocks = static_cast<int>((a.d + 127) / 128);
   const int items = m_blocks * a.splits;
   const int grid2 = items < num_sms ? items : num_sms;
-  decode_down_kernel<<<grid2, NUM_THREADS, K2_SMEM_BYTES, st>>>(a.tm_wd, a.tm_h, a.partial, a.counters, a.R, a.Y, a.y_bf16,
-                                                               a.n, a.d, m_blocks, a.splits, static_cast<int>(a.Ipad / BK),
-                                                               a.npad, a.status);
-  return cudaGetLastError();
+  return launch_pdl(decode_down_kernel, dim3(grid2), dim3(NUM_THREADS), K2_SMEM_BYTES, st, a.tm_wd, a.tm_h, a.partial, a.counters,
+                    a.R, a.Y, a.y_bf16, a.n, a.d, m_blocks, a.splits, static_cast<int>(a.Ipad / BK), a.npad, a.status);
 }
 
 }  // namespace mlpmoe

@@ -188,6 +188,8 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ 
                                                       float eps) {
   const int64_t t = static_cast<int64_t>(blockIdx.x) * (blockDim.x / 32) + threadIdx.x / 32;
   const int lane = threadIdx.x % 32;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may begin its set-up
+  asm volatile("griddepcontrol.wait;" ::: "memory");                // x written by the previous kernel is complete
   if (t >= n) return;
   const float4* row = reinterpret_cast<const float4*>(x + t * d);
   const int64_t nv = d / 4;
@@ -294,10 +296,8 @@ cudaError_t launch_fade(const FadeSeg* segs_host, int nseg, void* work, int elem
 cudaError_t launch_rmsnorm(const float* x, void* r, int64_t n, int64_t d, float eps, int out_elem_size, cudaStream_t st) {
   if (n == 0) return cudaSuccess;
   if (out_elem_size == 2)
-    rmsnorm_kernel<true><<<cdiv(n, 8), 256, 0, st>>>(x, r, n, d, eps);
-  else
-    rmsnorm_kernel<false><<<cdiv(n, 8), 256, 0, st>>>(x, r, n, d, eps);
-  return cudaGetLastError();
+    return launch_pdl(rmsnorm_kernel<true>, dim3(cdiv(n, 8)), dim3(256), 0, st, x, r, n, d, eps);
+  return launch_pdl(rmsnorm_kernel<false>, dim3(cdiv(n, 8)), dim3(256), 0, st, x, r, n, d, eps);
 }
 
 }  // namespace mlpmoe

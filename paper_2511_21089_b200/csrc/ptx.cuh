@@ -18,6 +18,14 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
   return t;
 }
 
+// ------------------------------------------- programmatic dependent launch --
+// wait: blocks until every kernel this launch depends on has completed and its writes are
+// visible (a no-op for a launch without the programmatic-serialization attribute).
+// launch_dependents: lets the next kernel in the stream start its own set-up early; that
+// kernel still waits, at its griddepcontrol.wait, for this grid to finish.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ------------------------------------------------------------------ mbarrier --
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));

@@ -65,6 +65,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_launch_dependents();          // the next kernel may begin its set-up
+  griddep_wait();                       // inputs written by earlier kernels are complete and visible
   const int num_tiles = num_m_blocks * num_n_blocks;
 
   if (warp == 0) {
@@ -185,9 +187,8 @@ cudaError_t launch_tc_gateup(const TcGateUpArgs& a, int num_sms, cudaStream_t st
   ep.status = a.status;
   const int tiles = m_blocks * n_blocks;
   const int grid = tiles < num_sms ? tiles : num_sms;
-  tc_gemm_kernel<GU_BN, GU_STAGES, EPI_SWIGLU><<<grid, NUM_THREADS, Cfg<GU_BN, GU_STAGES>::SMEM_BYTES, st>>>(
-      a.tm_x, a.tm_w, ep, m_blocks, n_blocks, k_blocks);
-  return cudaGetLastError();
+  return launch_pdl(tc_gemm_kernel<GU_BN, GU_STAGES, EPI_SWIGLU>, dim3(grid), dim3(NUM_THREADS),
+                    Cfg<GU_BN, GU_STAGES>::SMEM_BYTES, st, a.tm_x, a.tm_w, ep, m_blocks, n_blocks, k_blocks);
 }
 
 cudaError_t launch_tc_down(const TcDownArgs& a, int num_sms, cudaStream_t st) {
@@ -205,9 +206,8 @@ cudaError_t launch_tc_down(const TcDownArgs& a, int num_sms, cudaStream_t st) {
   ep.status = a.status;
   const int tiles = m_blocks * n_blocks;
   const int grid = tiles < num_sms ? tiles : num_sms;
-  tc_gemm_kernel<DN_BN, DN_STAGES, EPI_OUT><<<grid, NUM_THREADS, Cfg<DN_BN, DN_STAGES>::SMEM_BYTES, st>>>(
-      a.tm_h, a.tm_w, ep, m_blocks, n_blocks, k_blocks);
-  return cudaGetLastError();
+  return launch_pdl(tc_gemm_kernel<DN_BN, DN_STAGES, EPI_OUT>, dim3(grid), dim3(NUM_THREADS), Cfg<DN_BN, DN_STAGES>::SMEM_BYTES,
+                    st, a.tm_h, a.tm_w, ep, m_blocks, n_blocks, k_blocks);
 }
 
 }  // namespace mlpmoe

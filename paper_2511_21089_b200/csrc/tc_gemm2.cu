@@ -76,6 +76,8 @@ tc_pair_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
   cluster_sync_all();                   // both CTAs' barriers and TMEM exist before any remote signal
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_launch_dependents();          // the next kernel may begin its set-up
+  griddep_wait();                       // inputs written by earlier kernels are complete and visible
   const int num_tiles = num_m_pairs * num_n_blocks;
   const int first_tile = static_cast<int>(cluster_id_x());
   const int tile_step = static_cast<int>(cluster_count_x());
@@ -222,9 +224,8 @@ cudaError_t launch_tc_pair_gateup(const TcGateUpArgs& a, int num_sms, cudaStream
   ep.status = a.status;
   const int tiles = m_pairs * n_blocks;
   const int pairs = tiles < num_sms / 2 ? tiles : num_sms / 2;
-  tc_pair_gemm_kernel<EPI_SWIGLU><<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(a.tm_x, a.tm_w, a.tm_out, ep, m_pairs, n_blocks,
-                                                                            k_blocks, 256, OUT_TMA_STORE);
-  return cudaGetLastError();
+  return launch_pdl(tc_pair_gemm_kernel<EPI_SWIGLU>, dim3(2 * pairs), dim3(NUM_THREADS), SMEM_BYTES, st, a.tm_x, a.tm_w, a.tm_out,
+                    ep, m_pairs, n_blocks, k_blocks, 256, static_cast<int>(OUT_TMA_STORE));
 }
 
 cudaError_t launch_tc_pair_down(const TcDownArgs& a, int bn, int num_sms, cudaStream_t st) {
@@ -247,9 +248,8 @@ cudaError_t launch_tc_pair_down(const TcDownArgs& a, int bn, int num_sms, cudaSt
   int mode = OUT_DIRECT;
   if (!a.y_bf16 && a.R == nullptr) mode = OUT_TMA_STORE;
   else if (!a.y_bf16 && a.R == a.Y) mode = OUT_TMA_ADD;
-  tc_pair_gemm_kernel<EPI_OUT><<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(a.tm_h, a.tm_w, a.tm_out, ep, m_pairs, n_blocks,
-                                                                         k_blocks, bn, mode);
-  return cudaGetLastError();
+  return launch_pdl(tc_pair_gemm_kernel<EPI_OUT>, dim3(2 * pairs), dim3(NUM_THREADS), SMEM_BYTES, st, a.tm_h, a.tm_w, a.tm_out, ep,
+                    m_pairs, n_blocks, k_blocks, bn, mode);
 }
 
 }  // namespace mlpmoe
