@@ -51,6 +51,23 @@ def layer_inputs(layer: int, w):
     return bits, d_b, keep
 
 
+# DRAM traffic of one gate|up launch from the ncu capture summarised in
+# profiles/tc_pair_gemm_qwen_c2_2layers.md (dram__bytes_read.sum + dram__bytes_write.sum), valid
+# only while the kernel's sources are the ones that were profiled.
+GATEUP_TRAFFIC_BYTES = 20.70e6 + 0.12e6
+GATEUP_SOURCES = ("tc_gemm2.cu", "tc_common.cuh", "ptx.cuh")
+GATEUP_SOURCES_SHA = "b842eb5204afc5ef"
+
+
+def gateup_traffic():
+    import hashlib
+    h = hashlib.sha256()
+    for f in GATEUP_SOURCES:
+        with open(os.path.join(ROOT, "paper_2511_21089_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return GATEUP_TRAFFIC_BYTES if h.hexdigest()[:16] == GATEUP_SOURCES_SHA else None
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -289,7 +306,7 @@ def run_ours(args):
             achieved = float(np.mean(flops_gu)) / (gu_ms * 1e-3) / 1e12
             out["roofline"] = {"bound": "tensor", "kernel": "gate|up GEMM + SiLU*up epilogue (tcgen05)",
                                "achieved": achieved, "peak": pk["tflops_sustained"], "unit": "TFLOP/s",
-                               "frac": achieved / pk["tflops_sustained"], "traffic": None,
+                               "frac": achieved / pk["tflops_sustained"], "traffic": gateup_traffic(),
                                "peak_source": pk["source"] + " (sustained bf16 matmul)", "avg_launch_us": gu_ms * 1e3}
             out["kernels"] = {
                 "gate_up": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_total)},
