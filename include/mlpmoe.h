@@ -215,6 +215,36 @@ mlpmoe_status_t mlpmoe_set_timing(mlpmoe_handle_t h, int32_t enable);
 mlpmoe_status_t mlpmoe_get_timing(mlpmoe_handle_t h, double* ms, int64_t* launches);
 
 /* ------------------------------------------------------------------------- *
+ * Allocation-free variant (the paper has no counterpart: this is a deployment aid)
+ * ------------------------------------------------------------------------- */
+
+#define MLPMOE_STATIC_FADE_MAX_SLICES 256
+
+/*
+ * The masking step of mlpmoe_fade applied directly to caller-owned device buffers, without a
+ * layer handle and without allocating anything: for each slice i (m[i] contiguous elements of
+ * `dtype` at slices[i]) every entry with |w| <= (lo-th smallest |w|), lo = floor(s[i] (m[i] - 1))
+ * in exact arithmetic, is zeroed in place; s[i] = 0 leaves the slice untouched.  Pass one slice
+ * per (branch, projection) to reproduce mlpmoe_fade.
+ *
+ * For callers that cannot call cudaMalloc when they need this - a process whose device memory
+ * was handed to its own arena at start-up, or a path that must avoid cudaMalloc's device-wide
+ * synchronisation.  The scratch the selection needs (about 1.1 KB per slice) lives in a fixed
+ * array of about 275 KB inside the library image, present on every device that loads the
+ * library for the life of the process.  The call uses no cudaMalloc, cudaFree or other
+ * allocating routine.
+ *   slices, m, s   host arrays of length n_slices (slices holds device pointers).
+ *   n_slices       at most MLPMOE_STATIC_FADE_MAX_SLICES, else MLPMOE_ERR_UNSUPPORTED.
+ * The first call on each device looks up the array's device address (the device must be
+ * current); make that first call outside any stream capture.  All calls share the one array:
+ * each call re-initialises the part it uses, but two calls whose kernels overlap on the GPU
+ * (different streams, or different host threads) race on it - serialise them.  Synchronises
+ * `stream` before returning.
+ */
+mlpmoe_status_t mlpmoe_fade_buffers_static(void* const* slices, const int64_t* m, const double* s,
+                                           int32_t n_slices, mlpmoe_dtype_t dtype, void* stream);
+
+/* ------------------------------------------------------------------------- *
  * Host-only helpers: the scheduler's integer logic without any CUDA call
  * ------------------------------------------------------------------------- */
 

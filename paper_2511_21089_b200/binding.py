@@ -57,6 +57,7 @@ SIGNATURES = {
     "mlpmoe_status_string": (c_char_p, [c_int32]),
     "mlpmoe_set_timing": (c_int32, [c_void_p, c_int32]),
     "mlpmoe_get_timing": (c_int32, [c_void_p, POINTER(c_double), POINTER(c_int64)]),
+    "mlpmoe_fade_buffers_static": (c_int32, [POINTER(c_void_p), POINTER(c_int64), POINTER(c_double), c_int32, c_int32, c_void_p]),
     "mlpmoe_host_fade_position": (c_int32, [c_double, c_int64, POINTER(c_int64)]),
     "mlpmoe_host_fade_position_default": (c_int32, [c_int32, c_int32, c_int64, POINTER(c_int64)]),
     "mlpmoe_host_prune_alpha": (c_int32, [c_int32, POINTER(c_float), POINTER(c_uint8), c_int32, POINTER(c_float)]),
@@ -224,6 +225,20 @@ def mlpmoe_get_timing(h: int):
     cnt = (c_int64 * 3)()
     _check(lib.mlpmoe_get_timing(h, ms, cnt), "mlpmoe_get_timing")
     return list(ms), list(cnt)
+
+
+def mlpmoe_fade_buffers_static(slices: Sequence, s: Sequence[float], dtype: int = MLPMOE_BF16, stream=None) -> None:
+    """Mask caller-owned device buffers in place (one contiguous tensor per slice) with the library's
+    built-in scratch; allocates nothing.  `slices` are torch CUDA tensors or (address, n_elements) pairs."""
+    ptrs, sizes = [], []
+    for t in slices:
+        if isinstance(t, tuple):
+            ptrs.append(t[0]); sizes.append(t[1])
+        else:
+            ptrs.append(t.data_ptr()); sizes.append(t.numel())
+    n = len(ptrs)
+    _check(lib.mlpmoe_fade_buffers_static((c_void_p * n)(*ptrs), (c_int64 * n)(*sizes), (c_double * n)(*s), n, dtype,
+                                          _stream(stream)), "mlpmoe_fade_buffers_static")
 
 
 def mlpmoe_host_fade_position(s: float, m: int) -> int:
