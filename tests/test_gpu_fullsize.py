@@ -1,0 +1,158 @@
+"""Full-size parity runs on Llama-3-8B-shaped MLPs (d_model 4096, d_inter 14336), in the launch
+configurations the library uses at these sizes, against the oracle on sampled token rows
+(rows are independent, so the oracle runs exactly those rows):
+
+  config 3: one layer, B = 32 x 448, 8192 tokens, alpha ~ U(0.8, 1.2), Fractal Fade s_b = 0.9 b / B
+  config 4: 32-layer stack, B = 64 x 224, decode token counts 1 / 8 / 32 / 64, unpruned and
+            first-K pruning with K = 51
+  config 5: 32-layer stack, prefill, unequal seeded partitions, Compensated Pruning by ratio
+            (a sample of the sweep's corners: B = 4 / 128, tokens = 2048 / 16384)
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_21089_b200 import synth
+from tests.helpers import TOL_BF16, bits_of, dev_bf16, dev_f32, rel_err, stream_ptr
+
+pytestmark = pytest.mark.gpu
+
+D, I, L = 4096, 14336, 32
+
+
+def test_config3_fade_full_size(lib):
+    B, n = 32, 8192
+    d_b = synth.equal_partition(I, B)
+    bits = synth.layer_weights(3, 0, D, I, 0.02, bf16=True)
+    host = [synth.bf16_bits_to_f32(b) for b in bits]
+    alpha = synth.uniform_f64((synth.BASE_SEED, 3, 0, synth.T_ALPHA), B, 0.8, 1.2).astype(np.float32)
+    dev = [dev_bf16(b) for b in bits]
+    h = lib.mlpmoe_create(D, I, d_b, dev[0], dev[1], dev[2], alpha.tolist(), lib.MLPMOE_BF16, lib.MLPMOE_LAYOUT_PAPER, n, stream_ptr())
+    try:
+        lib.mlpmoe_fade(h, None, stream_ptr())
+        Fg, Fu = oracle.fade(host[0], host[1], d_b)
+        wg = torch.empty_like(dev[0]); wu = torch.empty_like(dev[1])
+        lib.mlpmoe_get_weights(h, wg, wu, None, stream_ptr())
+        torch.cuda.synchronize()
+        assert np.array_equal(synth.bf16_bits_to_f32(bits_of(wg)), Fg)          # masks bit-exact, 58.7 M entries each
+        assert np.array_equal(synth.bf16_bits_to_f32(bits_of(wu)), Fu)
+        nnz = lib.mlpmoe_nnz(h, B)
+        assert nnz == oracle.nnz_per_branch(Fg, Fu, host[2], d_b)
+        # sparsity rises with the branch index; branch 0 dense; about 43.6 % of gate+up zeroed at B = 32
+        frac = [1.0 - g / (D * 448) for g in nnz[0]]
+        assert frac[0] < 1e-3 and all(frac[b] < frac[b + 1] for b in range(B - 1))
+        assert abs(sum(frac) / B - 0.9 * (B - 1) / (2 * B)) < 5e-3
+        assert lib.mlpmoe_get_klist(h, B, I) == oracle.surviving_set(alpha, Fg, Fu, host[2], d_b)
+        xb = synth.f32_to_bf16_bits(synth.tokens(3, n, D))
+        xd = dev_bf16(xb)
+        y = torch.empty((n, D), dtype=torch.float32, device="cuda")
+        lib.mlpmoe_forward(h, xd, y, n, stream_ptr())
+        torch.cuda.synchronize()
+        assert lib.mlpmoe_get_status(h) == lib.MLPMOE_OK
+        rows = sorted(set([0, 127, 128, 255, 256, 4095, 4096, n - 1] + list(np.random.default_rng(3).integers(0, n, size=40))))
+        ref = oracle.mlpmoe_forward(synth.bf16_bits_to_f32(xb[rows]), Fg, Fu, host[2], d_b, alpha)
+        got = y.cpu().numpy()
+        assert np.isfinite(got).all()
+        assert rel_err(got[rows], ref) <= TOL_BF16
+    finally:
+        lib.mlpmoe_destroy(h)
+
+
+@pytest.fixture(scope="module")
+def llama_stack():
+    """Seeded bf16 weights of the 32 Llama-shaped layers: bit patterns on the host, tensors on the device."""
+    host_bits, dev = [], []
+    for l in range(L):
+        bits = synth.layer_weights(4, l, D, I, 0.02, bf16=True)
+        host_bits.append(bits)
+        dev.append([dev_bf16(b) for b in bits])
+    yield host_bits, dev
+    del dev
+    torch.cuda.empty_cache()
+
+
+class LazyLayers:
+    """Sequence of oracle layer tuples that widens one layer's weights at a time."""
+
+    def __init__(self, host_bits, d_b, alphas):
+        self.host_bits, self.d_b, self.alphas = host_bits, d_b, alphas
+
+    def __iter__(self):
+        for bits, alpha in zip(self.host_bits, self.alphas):
+            yield (*[synth.bf16_bits_to_f32(b) for b in bits], self.d_b, alpha)
+
+
+def make_handles(lib, dev, d_b, max_tokens, prune=None):
+    handles = []
+    for l in range(L):
+        h = lib.mlpmoe_create(D, I, d_b, dev[l][0], dev[l][1], dev[l][2], None, lib.MLPMOE_BF16, lib.MLPMOE_LAYOUT_PAPER,
+                              max_tokens, stream_ptr())
+        if handles:
+            lib.mlpmoe_share_workspace(h, handles[0])
+        handles.append(h)
+        if prune is not None:
+            prune(l, h)
+    torch.cuda.synchronize()
+    return handles
+
+
+def destroy(lib, handles):
+    for h in handles[1:] + handles[:1]:
+        lib.mlpmoe_destroy(h)
+
+
+def test_config4_decode_stack(lib, llama_stack):
+    host_bits, dev = llama_stack
+    B = 64
+    d_b = synth.equal_partition(I, B)
+    x = synth.tokens(4, 64, D)
+    handles = make_handles(lib, dev, d_b, 64)
+    try:
+        for K in (None, 51):
+            if K is not None:
+                for h in handles:
+                    lib.mlpmoe_prune_first_k(h, K, stream_ptr())
+                alpha = oracle.prune_alpha([1.0] * B, oracle.first_k_keep(B, K))
+                assert lib.mlpmoe_get_active_neurons(handles[0]) == K * 224
+                assert lib.mlpmoe_get_klist(handles[-1], B, I) == (list(range(K)), [(224 * b, 224) for b in range(K)])
+            else:
+                alpha = [1.0] * B
+            ref = oracle.stack_forward(x, LazyLayers(host_bits, d_b, [alpha] * L), bf16_activations=True)
+            for n in (1, 8, 32, 64):
+                xd = dev_f32(x[:n])
+                lib.mlpmoe_stack_forward(handles, xd, n, 1e-6, stream_ptr())
+                torch.cuda.synchronize()
+                assert rel_err(xd.cpu().numpy(), ref[:n]) <= TOL_BF16, (K, n)
+            assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
+    finally:
+        destroy(lib, handles)
+
+
+@pytest.mark.parametrize("B,n,ratio", [(128, 2048, 0.4), (4, 16384, 0.1), (16, 2048, 0.2)])
+def test_config5_prefill_sweep_corners(lib, llama_stack, B, n, ratio):
+    host_bits, dev = llama_stack
+    d_b = synth.random_partition((synth.BASE_SEED, 5, B, synth.T_PARTITION), I, B, 64)
+    n_drop = synth.n_drop_for_ratio(B, ratio)
+    keeps = [synth.keep_set((synth.BASE_SEED, 5, B, l, synth.T_KEEP), B, n_drop) for l in range(L)]
+    alphas = [oracle.prune_alpha([1.0] * B, k) for k in keeps]
+    handles = make_handles(lib, dev, d_b, n, prune=lambda l, h: lib.mlpmoe_prune(h, keeps[l], True, stream_ptr()))
+    try:
+        offs = oracle.branch_offsets(d_b)
+        for l in (0, L - 1):
+            kept = [b for b in range(B) if keeps[l][b]]
+            assert lib.mlpmoe_get_klist(handles[l], B, I) == (kept, [(offs[b], d_b[b]) for b in kept])
+            assert np.array_equal(lib.mlpmoe_get_alpha(handles[l], B).view(np.uint32),
+                                  np.array(alphas[l]).astype(np.float32).view(np.uint32))
+        x = synth.tokens(5, n, D, stream=B)
+        xd = dev_f32(x)
+        lib.mlpmoe_stack_forward(handles, xd, n, 1e-6, stream_ptr())
+        torch.cuda.synchronize()
+        rows = sorted(set([0, 255, 256, n - 1] + list(np.random.default_rng(B).integers(0, n, size=8))))
+        ref = oracle.stack_forward(x[rows], LazyLayers(host_bits, d_b, alphas), bf16_activations=True)
+        got = xd.cpu().numpy()
+        assert np.isfinite(got).all()
+        assert rel_err(got[rows], ref) <= TOL_BF16
+        assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
+    finally:
+        destroy(lib, handles)
