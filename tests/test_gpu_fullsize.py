@@ -97,6 +97,36 @@ def make_handles(lib, dev, d_b, max_tokens, prune=None):
     return handles
 
 
+def layer_rms(inputs, out):
+    """RMS of every layer's own contribution y_l = x_{l+1} - x_l in the oracle's run."""
+    xs = list(inputs) + [out]
+    return [float(np.sqrt(np.mean((xs[l + 1] - xs[l]) ** 2))) for l in range(len(inputs))]
+
+
+def check_layers_one_by_one(lib, handles, which, inputs, out, n_launch):
+    """Each GPU layer, fed the oracle's input of that layer, must reproduce the oracle's contribution
+    of that layer within the layer tolerance.  The first rows of an n_launch-row batch carry the
+    sampled rows (the rest are zero), so the kernels run in their n_launch-token configuration."""
+    xs = list(inputs) + [out]
+    rows = xs[0].shape[0]
+    for l in which:
+        xin = np.zeros((n_launch, D), dtype=np.float32)
+        xin[:rows] = xs[l].astype(np.float32)
+        xd = dev_f32(xin)
+        lib.mlpmoe_stack_forward([handles[l]], xd, n_launch, 1e-6, stream_ptr())
+        torch.cuda.synchronize()
+        got = xd.cpu().numpy()[:rows].astype(np.float64) - xin[:rows].astype(np.float64)
+        assert rel_err(got, xs[l + 1] - xs[l]) <= TOL_BF16, l
+
+
+def stack_tolerance(inputs, out):
+    """End-to-end bound for a deep stack, as a multiple of RMS(output): every layer's contribution
+    may be off by TOL_BF16 * RMS(y_l); the stack output is the sum of the contributions, so to first
+    order its error is bounded by the sum of those, and the later layers' response to the perturbed
+    stream (damped by RMSNorm, since the stream's RMS grows with depth) is allowed the same again."""
+    return 2.0 * TOL_BF16 * sum(layer_rms(inputs, out)) / float(np.sqrt(np.mean(out ** 2)))
+
+
 def destroy(lib, handles):
     for h in handles[1:] + handles[:1]:
         lib.mlpmoe_destroy(h)
@@ -118,12 +148,17 @@ def test_config4_decode_stack(lib, llama_stack):
                 assert lib.mlpmoe_get_klist(handles[-1], B, I) == (list(range(K)), [(224 * b, 224) for b in range(K)])
             else:
                 alpha = [1.0] * B
-            ref = oracle.stack_forward(x, LazyLayers(host_bits, d_b, [alpha] * L), bf16_activations=True)
+            ref, inputs = oracle.stack_forward(x, LazyLayers(host_bits, d_b, [alpha] * L), bf16_activations=True,
+                                               return_layer_inputs=True)
+            check_layers_one_by_one(lib, handles, range(L), inputs, ref, 64)
+            check_layers_one_by_one(lib, handles, (0, L - 1), [v[:1] for v in inputs], ref[:1], 1)
+            tol = stack_tolerance(inputs, ref)
+            assert tol < 0.25
             for n in (1, 8, 32, 64):
                 xd = dev_f32(x[:n])
                 lib.mlpmoe_stack_forward(handles, xd, n, 1e-6, stream_ptr())
                 torch.cuda.synchronize()
-                assert rel_err(xd.cpu().numpy(), ref[:n]) <= TOL_BF16, (K, n)
+                assert rel_err(xd.cpu().numpy(), ref[:n]) <= tol, (K, n)
             assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
     finally:
         destroy(lib, handles)
@@ -149,10 +184,12 @@ def test_config5_prefill_sweep_corners(lib, llama_stack, B, n, ratio):
         lib.mlpmoe_stack_forward(handles, xd, n, 1e-6, stream_ptr())
         torch.cuda.synchronize()
         rows = sorted(set([0, 255, 256, n - 1] + list(np.random.default_rng(B).integers(0, n, size=8))))
-        ref = oracle.stack_forward(x[rows], LazyLayers(host_bits, d_b, alphas), bf16_activations=True)
+        ref, inputs = oracle.stack_forward(x[rows], LazyLayers(host_bits, d_b, alphas), bf16_activations=True,
+                                           return_layer_inputs=True)
         got = xd.cpu().numpy()
         assert np.isfinite(got).all()
-        assert rel_err(got[rows], ref) <= TOL_BF16
+        assert rel_err(got[rows], ref) <= stack_tolerance(inputs, ref)
+        check_layers_one_by_one(lib, handles, (0, L // 2, L - 1), inputs, ref, n)
         assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
     finally:
         destroy(lib, handles)
