@@ -30,7 +30,6 @@ if ROOT not in sys.path:
 
 from paper_2511_21089_b200 import synth  # noqa: E402
 
-CFG = 2
 METRIC = "mlpmoe_mlp_tokens_per_s"
 UNIT = "tokens/s"
 WORKLOAD = ("configs[1]: 24-layer MLP-only stack, Qwen2.5-0.5B shapes (d_model=896, d_inter=4864), bf16, "
@@ -38,17 +37,54 @@ WORKLOAD = ("configs[1]: 24-layer MLP-only stack, Qwen2.5-0.5B shapes (d_model=8
             "RMSNorm + residual, 4096 tokens")
 
 
-def workload(layers=None):
-    c = synth.CONFIGS[CFG]
-    return dict(d=c["d_model"], I=c["d_inter"], B=c["B"], n=c["n"], L=layers or c["layers"], n_drop=c["n_drop"])
+def workload(layers=None, name="qwen_stack", tokens=None, branches=None, ratio=0.0, prune_k=None):
+    """The default (and only driver-run) workload is the 24-layer Qwen-shaped stack; the others are
+    the remaining configurations, for measurement of the decode and Llama-shaped prefill paths."""
+    if name == "qwen_stack":
+        c = synth.CONFIGS[2]
+        return dict(name=name, cfg=2, d=c["d_model"], I=c["d_inter"], B=c["B"], n=tokens or c["n"], L=layers or c["layers"],
+                    n_drop=c["n_drop"], stack=True, label=WORKLOAD)
+    c = synth.CONFIGS[4]
+    d, I = c["d_model"], c["d_inter"]
+    if name == "llama_decode":
+        n = tokens or 64
+        return dict(name=name, cfg=4, d=d, I=I, B=64, n=n, L=layers or 32, prune_k=prune_k, stack=True,
+                    label=f"configs[3]: 32-layer Llama-3-8B-shaped MLP stack, bf16, B=64 equal slices, decode, {n} tokens, "
+                          + (f"first-K pruning K={prune_k}" if prune_k else "no pruning"))
+    if name == "llama_layer_fade":
+        n = tokens or 8192
+        return dict(name=name, cfg=3, d=d, I=I, B=32, n=n, L=1, stack=False, fade=True,
+                    label=f"configs[2]: single Llama-3-8B-shaped layer, bf16, B=32, Fractal Fade s_b=0.9b/B, alpha~U(0.8,1.2), {n} tokens")
+    if name == "llama_prefill":
+        n, B = tokens or 2048, branches or 16
+        return dict(name=name, cfg=5, d=d, I=I, B=B, n=n, L=layers or 32, ratio=ratio, stack=True,
+                    label=f"configs[4]: 32-layer Llama-3-8B-shaped MLP stack, bf16, B={B} unequal slices, {n} tokens, "
+                          f"Compensated Pruning ratio {ratio}")
+    raise ValueError(name)
 
 
 def layer_inputs(layer: int, w):
-    """Seeded weights (bf16 bit patterns), partition and keep set of one layer."""
-    bits = synth.layer_weights(CFG, layer, w["d"], w["I"], 0.02, bf16=True)
-    d_b = synth.equal_partition(w["I"], w["B"])
-    keep = synth.keep_set((synth.BASE_SEED, CFG, layer, synth.T_KEEP), w["B"], w["n_drop"])
-    return bits, d_b, keep
+    """Seeded inputs of one layer: (weights as bf16 bit patterns, partition, alpha or None, keep mask or None)."""
+    cfg, B = w["cfg"], w["B"]
+    wcfg = 4 if cfg == 5 else cfg          # the prefill sweep runs on the decode configuration's weights
+    bits = synth.layer_weights(wcfg, layer, w["d"], w["I"], 0.02, bf16=True)
+    alpha, keep = None, None
+    if cfg == 2:
+        d_b = synth.equal_partition(w["I"], B)
+        keep = synth.keep_set((synth.BASE_SEED, cfg, layer, synth.T_KEEP), B, w["n_drop"])
+    elif cfg == 3:
+        d_b = synth.equal_partition(w["I"], B)
+        alpha = [float(a) for a in synth.uniform_f64((synth.BASE_SEED, 3, layer, synth.T_ALPHA), B, 0.8, 1.2).astype(np.float32)]
+    elif cfg == 4:
+        d_b = synth.equal_partition(w["I"], B)
+        if w.get("prune_k"):
+            keep = [b < w["prune_k"] for b in range(B)]
+    else:
+        d_b = synth.random_partition((synth.BASE_SEED, 5, B, synth.T_PARTITION), w["I"], B, 64)
+        n_drop = synth.n_drop_for_ratio(B, w["ratio"])
+        if n_drop:
+            keep = synth.keep_set((synth.BASE_SEED, 5, B, layer, synth.T_KEEP), B, n_drop)
+    return bits, d_b, alpha, keep
 
 
 # DRAM traffic of one gate|up launch from the ncu capture summarised in
@@ -83,7 +119,7 @@ def oracle_layers(w):
     import oracle
     layers = []
     for l in range(w["L"]):
-        bits, d_b, keep = layer_inputs(l, w)
+        bits, d_b, alpha, keep = layer_inputs(l, w)
         host = [synth.bf16_bits_to_f32(b) for b in bits]
         layers.append((host[0], host[1], host[2], d_b, oracle.prune_alpha([1.0] * w["B"], keep)))
     return layers
@@ -104,7 +140,7 @@ def time_oracle(w, rows: int, steps: int, warmup: int, layers=None):
     import oracle
     if layers is None:
         layers = oracle_layers(w)
-    x = synth.tokens(CFG, w["n"], w["d"])[:rows]
+    x = synth.tokens(w["cfg"], w["n"], w["d"])[:rows]
     for _ in range(warmup):
         oracle.stack_forward(x, layers, bf16_activations=True)
     t0 = time.perf_counter()
@@ -197,16 +233,19 @@ def run_ours(args):
         dist.barrier()
     from paper_2511_21089_b200 import binding as lib
 
-    w = workload(args.layers)
+    w = workload(args.layers, args.workload, args.tokens, args.branches, args.ratio, args.prune_k)
     n, d, L = w["n"], w["d"], w["L"]
     stream = torch.cuda.current_stream()
     st = stream.cuda_stream
     layers, active = [], []
     for l in range(L):
-        bits, d_b, keep = layer_inputs(l, w)
+        bits, d_b, alpha, keep = layer_inputs(l, w)
         dev = [torch.from_numpy(b.view(np.int16)).view(torch.bfloat16).cuda() for b in bits]
-        h = lib.mlpmoe_create(d, w["I"], d_b, dev[0], dev[1], dev[2], None, lib.MLPMOE_BF16, lib.MLPMOE_LAYOUT_PAPER, n, st)
-        lib.mlpmoe_prune(h, keep, True, st)
+        h = lib.mlpmoe_create(d, w["I"], d_b, dev[0], dev[1], dev[2], alpha, lib.MLPMOE_BF16, lib.MLPMOE_LAYOUT_PAPER, n, st)
+        if w.get("fade"):
+            lib.mlpmoe_fade(h, None, st)
+        if keep is not None:
+            lib.mlpmoe_prune(h, keep, True, st)
         if layers:
             lib.mlpmoe_share_workspace(h, layers[0])
         layers.append(h)
@@ -214,14 +253,32 @@ def run_ours(args):
         del dev
     torch.cuda.synchronize()
 
-    x0_host = torch.from_numpy(synth.tokens(CFG, n, d, stream=rank)).pin_memory()     # each rank its own batch
+    x_f32 = synth.tokens(w["cfg"], n, d, stream=rank)                                 # each rank its own batch
     y_host = torch.empty((n, d), dtype=torch.float32).pin_memory()
-    x0 = x0_host.cuda()
-    xw = torch.empty_like(x0)
+    if w["stack"]:
+        x0_host = torch.from_numpy(x_f32).pin_memory()
+        x0 = x0_host.cuda()
+        xw = torch.empty_like(x0)
 
-    def step():
-        xw.copy_(x0, non_blocking=True)          # fresh residual stream; inputs already resident in HBM
-        lib.mlpmoe_stack_forward(layers, xw, n, 1e-6, st)
+        def step():
+            xw.copy_(x0, non_blocking=True)      # fresh residual stream; inputs already resident in HBM
+            lib.mlpmoe_stack_forward(layers, xw, n, 1e-6, st)
+
+        def step_host():
+            lib.mlpmoe_stack_forward_host(layers, x0_host, y_host, n, 1e-6, st)
+        in_bytes = n * d * 4
+    else:
+        xb = synth.f32_to_bf16_bits(x_f32)
+        x0_host = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()
+        x0 = x0_host.cuda()
+        xw = torch.empty((n, d), dtype=torch.float32, device="cuda")
+
+        def step():
+            lib.mlpmoe_forward(layers[0], x0, xw, n, st)
+
+        def step_host():
+            lib.mlpmoe_forward_host(layers[0], x0_host, y_host, n, st)
+        in_bytes = n * d * 2
 
     def barrier():
         if world > 1:
@@ -268,12 +325,12 @@ def run_ours(args):
 
     # end to end through the host-buffer entry point: H2D of x and D2H of y inside the timed region
     for _ in range(2):
-        lib.mlpmoe_stack_forward_host(layers, x0_host, y_host, n, 1e-6, st)
+        step_host()
     barrier()
     e2e_steps = max(3, min(args.steps, 10))
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        lib.mlpmoe_stack_forward_host(layers, x0_host, y_host, n, 1e-6, st)     # synchronises the stream itself
+        step_host()                                  # synchronises the stream itself
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
     if not np.isfinite(y_host.numpy()).all():
         raise RuntimeError("non-finite output")
@@ -289,34 +346,48 @@ def run_ours(args):
         pk = peaks()
         flops_gu = [4.0 * n * d * a for a in active]              # algorithmic FLOPs of each gate|up launch
         flops_dn = [2.0 * n * d * a for a in active]
+        wbytes_gu = [2.0 * d * a * 2 for a in active]             # weight bytes each gate|up launch must stream
+        wbytes_dn = [1.0 * d * a * 2 for a in active]
+        default = w["name"] == "qwen_stack" and L == synth.CONFIGS[2]["layers"] and n == synth.CONFIGS[2]["n"]
+        weights_gb = (sum(wbytes_gu) + sum(wbytes_dn)) / 1e9
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
-            "config": {"workload": WORKLOAD if L == synth.CONFIGS[CFG]["layers"] else WORKLOAD + f" [REDUCED to {L} layers]", "l2": "inputs larger than L2: each step streams 0.47 GB of distinct weights",
+            "config": {"workload": w["label"] if default or w["name"] != "qwen_stack" else w["label"] + f" [REDUCED to {L} layers, {n} tokens]",
+                       "l2": f"inputs larger than L2: each step streams {weights_gb:.2f} GB of distinct weights",
                        "surviving_neurons_per_layer": int(np.mean(active)), "tokens_per_rank": n},
             "clocks": clocks,
-            "e2e": {"value": world * n / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": n * d * 4,
+            "e2e": {"value": world * n / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": in_bytes,
                     "d2h_bytes_per_step": n * d * 4, "ms_per_step": e2e_ms},
             "gpu_launches": int(launches),
             "tflops": (sum(flops_gu) + sum(flops_dn)) / (ms_step * 1e-3) / 1e12,
+            "weight_gbs": weights_gb / (ms_step * 1e-3),
         }
         if kcnt[0] > 0:
             gu_ms = kms[0] / kcnt[0]
-            achieved = float(np.mean(flops_gu)) / (gu_ms * 1e-3) / 1e12
-            out["roofline"] = {"bound": "tensor", "kernel": "gate|up GEMM + SiLU*up epilogue (tcgen05)",
-                               "achieved": achieved, "peak": pk["tflops_sustained"], "unit": "TFLOP/s",
-                               "frac": achieved / pk["tflops_sustained"], "traffic": gateup_traffic(),
-                               "peak_source": pk["source"] + " (sustained bf16 matmul)", "avg_launch_us": gu_ms * 1e3}
+            dn_ms = kms[1] / max(kcnt[1], 1)
+            if n > 64:
+                achieved = float(np.mean(flops_gu)) / (gu_ms * 1e-3) / 1e12
+                out["roofline"] = {"bound": "tensor", "kernel": "gate|up GEMM + SiLU*up epilogue (tcgen05)",
+                                   "achieved": achieved, "peak": pk["tflops_sustained"], "unit": "TFLOP/s",
+                                   "frac": achieved / pk["tflops_sustained"], "traffic": gateup_traffic() if default else None,
+                                   "peak_source": pk["source"] + " (sustained bf16 matmul)", "avg_launch_us": gu_ms * 1e3}
+            else:
+                achieved = float(np.mean(wbytes_gu)) / (gu_ms * 1e-3) / 1e9
+                out["roofline"] = {"bound": "hbm", "kernel": "decode gate|up weight-streaming kernel (TMA ring + tcgen05)",
+                                   "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
+                                   "traffic": None, "peak_source": pk["source"] + " (copy bandwidth)", "avg_launch_us": gu_ms * 1e3}
             out["kernels"] = {
-                "gate_up": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_total)},
-                "down": {"avg_us": kms[1] / max(kcnt[1], 1) * 1e3, "launches": int(kcnt[1]), "share": float(kms[1] / ms_total),
-                         "tflops": float(np.mean(flops_dn)) / (kms[1] / max(kcnt[1], 1) * 1e-3) / 1e12},
+                "gate_up": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_total),
+                            "tflops": float(np.mean(flops_gu)) / (gu_ms * 1e-3) / 1e12, "weight_gbs": float(np.mean(wbytes_gu)) / (gu_ms * 1e-3) / 1e9},
+                "down": {"avg_us": dn_ms * 1e3, "launches": int(kcnt[1]), "share": float(kms[1] / ms_total),
+                         "tflops": float(np.mean(flops_dn)) / (dn_ms * 1e-3) / 1e12, "weight_gbs": float(np.mean(wbytes_dn)) / (dn_ms * 1e-3) / 1e9},
                 "rmsnorm": {"avg_us": kms[2] / max(kcnt[2], 1) * 1e3, "launches": int(kcnt[2]), "share": float(kms[2] / ms_total)},
             }
         else:
             out["roofline"] = None
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and w["name"] == "qwen_stack":
             rows = 512
             tps, dt = time_oracle(w, rows, 3, 1)
             out["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
@@ -337,6 +408,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--layers", type=int, default=None, help="fewer layers of the same stack (profiling captures only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen_stack", choices=["qwen_stack", "llama_decode", "llama_layer_fade", "llama_prefill"],
+                    help="the driver runs the default; the others measure the remaining configurations")
+    ap.add_argument("--tokens", type=int, default=None)
+    ap.add_argument("--branches", type=int, default=None)
+    ap.add_argument("--ratio", type=float, default=0.0)
+    ap.add_argument("--prune-k", type=int, default=None)
     ap.add_argument("--kernel-events", type=int, default=1, help="record per-kernel CUDA events in the timed region")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
