@@ -258,6 +258,7 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
   if (n == 0) return MLPMOE_OK;
   if (!x || !y || n > h->max_tokens || !aligned16(x) || !aligned16(y) || (residual && !aligned16(residual)))
     return MLPMOE_ERR_INVALID_ARG;
+  pdl_overlap_enabled() = !h->timing;
   if (y_dtype != MLPMOE_FP32 && !(y_dtype == MLPMOE_BF16 && h->dtype == MLPMOE_BF16)) return MLPMOE_ERR_UNSUPPORTED;
   if (h->dtype == MLPMOE_FP32) {
     float* H = static_cast<float*>(h->ws->H);
@@ -541,6 +542,7 @@ mlpmoe_status_t mlpmoe_rmsnorm(const float* x, void* r, int64_t n_tokens, int64_
   if (n_tokens < 0 || d_model <= 0 || d_model % 4 != 0) return MLPMOE_ERR_INVALID_ARG;
   if (n_tokens == 0) return MLPMOE_OK;
   if (!x || !r || !aligned16(x) || !aligned16(r)) return MLPMOE_ERR_INVALID_ARG;
+  pdl_overlap_enabled() = true;
   CK(launch_rmsnorm(x, r, n_tokens, d_model, eps, out_dtype == MLPMOE_BF16 ? 2 : 4, static_cast<cudaStream_t>(stream)));
   return MLPMOE_OK;
 }
@@ -554,6 +556,7 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   for (int l = 0; l < n_layers; ++l) {
     mlpmoe_layer_s* h = layers[l];
+    pdl_overlap_enabled() = !h->timing;
     const long e0 = rec_event(h, st);
     CK(launch_rmsnorm(x, h->ws->xnorm, n, h->d, eps, h->elem_size, st));
     const long e1 = rec_event(h, st);

@@ -11,6 +11,13 @@ namespace mlpmoe {
 // Launch with programmatic stream serialization: the kernel may begin (set-up only) while its
 // predecessor in the stream drains; every kernel launched this way executes griddepcontrol.wait
 // before it touches global memory.
+// Overlap is switched off (plain stream order) while a handle records per-kernel CUDA events:
+// an event between two overlapped kernels would not mark the end of the first one.
+inline bool& pdl_overlap_enabled() {
+  static thread_local bool on = true;
+  return on;
+}
+
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
   cudaLaunchConfig_t cfg = {};
@@ -20,7 +27,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[0].val.programmaticStreamSerializationAllowed = pdl_overlap_enabled() ? 1 : 0;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
