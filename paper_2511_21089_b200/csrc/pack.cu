@@ -194,13 +194,50 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ 
   const float4* row = reinterpret_cast<const float4*>(x + t * d);
   const int64_t nv = d / 4;
   float ss = 0.f;
+#pragma unroll 8
   for (int64_t v = lane; v < nv; v += 32) {
     const float4 a = row[v];
     ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
   }
   for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
   const float inv = 1.0f / sqrtf(ss / static_cast<float>(d) + eps);
+#pragma unroll 8
   for (int64_t v = lane; v < nv; v += 32) {
+    const float4 a = row[v];
+    if (OUT_BF16) {
+      uint2 o;
+      o.x = static_cast<uint32_t>(f32_to_bf16_rn(a.x * inv)) | (static_cast<uint32_t>(f32_to_bf16_rn(a.y * inv)) << 16);
+      o.y = static_cast<uint32_t>(f32_to_bf16_rn(a.z * inv)) | (static_cast<uint32_t>(f32_to_bf16_rn(a.w * inv)) << 16);
+      reinterpret_cast<uint2*>(static_cast<uint16_t*>(r) + t * d)[v] = o;
+    } else {
+      reinterpret_cast<float4*>(static_cast<float*>(r) + t * d)[v] = make_float4(a.x * inv, a.y * inv, a.z * inv, a.w * inv);
+    }
+  }
+}
+
+// Few rows (decode): one 256-thread block per row, so that a row's loads are all in flight at once.
+template <bool OUT_BF16>
+__global__ void __launch_bounds__(256) rmsnorm_block_kernel(const float* __restrict__ x, void* __restrict__ r, int64_t n,
+                                                            int64_t d, float eps) {
+  const int64_t t = blockIdx.x;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const float4* row = reinterpret_cast<const float4*>(x + t * d);
+  const int64_t nv = d / 4;
+  float ss = 0.f;
+  for (int64_t v = threadIdx.x; v < nv; v += blockDim.x) {
+    const float4 a = row[v];
+    ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+  }
+  __shared__ float red[8];
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+  if (threadIdx.x % 32 == 0) red[threadIdx.x / 32] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tot += red[i];
+  const float inv = 1.0f / sqrtf(tot / static_cast<float>(d) + eps);
+  for (int64_t v = threadIdx.x; v < nv; v += blockDim.x) {
     const float4 a = row[v];
     if (OUT_BF16) {
       uint2 o;
@@ -295,6 +332,11 @@ cudaError_t launch_fade(const FadeSeg* segs_host, int nseg, void* work, int elem
 
 cudaError_t launch_rmsnorm(const float* x, void* r, int64_t n, int64_t d, float eps, int out_elem_size, cudaStream_t st) {
   if (n == 0) return cudaSuccess;
+  if (n <= 1024) {     // not enough rows to fill the GPU with one warp per row
+    if (out_elem_size == 2)
+      return launch_pdl(rmsnorm_block_kernel<true>, dim3(static_cast<unsigned>(n)), dim3(256), 0, st, x, r, n, d, eps);
+    return launch_pdl(rmsnorm_block_kernel<false>, dim3(static_cast<unsigned>(n)), dim3(256), 0, st, x, r, n, d, eps);
+  }
   if (out_elem_size == 2)
     return launch_pdl(rmsnorm_kernel<true>, dim3(cdiv(n, 8)), dim3(256), 0, st, x, r, n, d, eps);
   return launch_pdl(rmsnorm_kernel<false>, dim3(cdiv(n, 8)), dim3(256), 0, st, x, r, n, d, eps);

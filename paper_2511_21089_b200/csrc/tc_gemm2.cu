@@ -195,8 +195,11 @@ cudaError_t tc_pair_init() {
   return cudaFuncSetAttribute(tc_pair_gemm_kernel<EPI_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
 }
 
-// Width of the down-projection tile: the multiple of 32 (64..256) that minimises
-// waves x width, i.e. the tensor-core time of the busiest CTA pair; ties go to the wider tile.
+// Width of the down-projection tile (a multiple of 32, 64..256): the one that minimises
+// waves x (time of one K-step), where a K-step costs the larger of its tensor-core time
+// (2 x width cycles for a 256 x width x 64 step) and the time to fill one CTA's stage from L2
+// (16 KB of A + width/2 rows of B at about 50 bytes per cycle per SM, the rate these kernels
+// see).  Narrow tiles need fewer waves but re-read A more often; ties go to the wider tile.
 int tc_pair_down_bn(int64_t n, int64_t d, int num_sms) {
   const int64_t pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
   const int64_t m_pairs = (n + 255) / 256;
@@ -204,7 +207,10 @@ int tc_pair_down_bn(int64_t n, int64_t d, int num_sms) {
   int64_t best_cost = -1;
   for (int bn = 256; bn >= 64; bn -= 32) {
     const int64_t tiles = m_pairs * ((d + bn - 1) / bn);
-    const int64_t cost = ((tiles + pairs - 1) / pairs) * bn;
+    const int64_t mma_cycles = 2 * bn;
+    const int64_t fill_cycles = (A_BYTES + (bn / 2) * BK * 2) / 50;
+    const int64_t step = mma_cycles > fill_cycles ? mma_cycles : fill_cycles;
+    const int64_t cost = ((tiles + pairs - 1) / pairs) * step;
     if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
   }
   return best;
