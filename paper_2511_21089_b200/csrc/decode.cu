@@ -174,8 +174,8 @@ decode_gateup_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 decode_down_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_constant__ CUtensorMap tm_h,
-                   float* __restrict__ partial, uint32_t* __restrict__ counters, const float* __restrict__ R,
-                   void* __restrict__ Y, int y_bf16, int64_t n, int64_t d, int num_m_blocks, int splits,
+                   float* __restrict__ partial, uint32_t* __restrict__ counters, const float* R,
+                   void* Y, int y_bf16, int64_t n, int64_t d, int num_m_blocks, int splits,
                    int total_k_blocks, int npad, uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align_1024(smem_raw);
@@ -309,13 +309,18 @@ decode_down_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_const
               }
             }
           }
+          // all residual loads first, then all stores: R may alias Y (in-place residual stream), and a
+          // load placed after a store to a possibly aliasing address would wait for it
+          if (R != nullptr) {
+#pragma unroll
+            for (int t = 0; t < MAXN; ++t)
+              if (t < n) accv[t] += __ldcg(R + static_cast<int64_t>(t) * d + m);
+          }
 #pragma unroll
           for (int t = 0; t < MAXN; ++t) {
             if (t < n) {
-              float o = accv[t];
-              if (R != nullptr) o += R[static_cast<int64_t>(t) * d + m];
-              if (y_bf16) static_cast<__nv_bfloat16*>(Y)[static_cast<int64_t>(t) * d + m] = __float2bfloat16_rn(o);
-              else static_cast<float*>(Y)[static_cast<int64_t>(t) * d + m] = o;
+              if (y_bf16) static_cast<__nv_bfloat16*>(Y)[static_cast<int64_t>(t) * d + m] = __float2bfloat16_rn(accv[t]);
+              else static_cast<float*>(Y)[static_cast<int64_t>(t) * d + m] = accv[t];
             }
           }
         }
