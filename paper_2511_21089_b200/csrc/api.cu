@@ -172,6 +172,8 @@ struct mlpmoe_layer_s {
   void* fade_work = nullptr;
   float* partial = nullptr;
   uint32_t* counters = nullptr;
+  uint32_t* block_done = nullptr;                           // [2 x ceil(max_tokens / 256)] gate|up completion counters
+  int64_t max_blocks = 0;
   int max_splits = 1;
   uint32_t* status = nullptr;
   int64_t launches = 0;
@@ -206,7 +208,7 @@ void free_layer(mlpmoe_layer_s* h) {
   cudaFree(h->Wg_c); cudaFree(h->Wu_c); cudaFree(h->Wd_c);
   cudaFree(h->Wgu); cudaFree(h->WdT);
   cudaFree(h->scale); cudaFree(h->src_row); cudaFree(h->row_nnz);
-  cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->status);
+  cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->block_done); cudaFree(h->status);
   ws_release(h->ws);
   delete h;
 }
@@ -304,39 +306,58 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
     h->launches += 2;
     return MLPMOE_OK;
   }
-  // n > 128: CTA pairs (256-token tiles); 65..128 tokens: one CTA per tile
-  const bool pair = n > 128;
+  if (n > 128) {
+    // one fused CTA-pair kernel: gate|up tiles, then down tiles
+    TcLayerArgs a;
+    a.bn = tc_layer_down_bn(n, h->d, h->num_sms);
+    if (!make_tmap(&a.tm_x, x, h->d, n, h->d, 128)) return MLPMOE_ERR_CUDA;
+    a.tm_wgu = h->tm_wgu_pair;
+    if (!make_tmap(&a.tm_h_st, h->ws->H, h->Ipad, n, h->Ipad, 32)) return MLPMOE_ERR_CUDA;
+    if (!make_tmap(&a.tm_h_ld, h->ws->H, h->Ipad, n, h->Ipad, 128)) return MLPMOE_ERR_CUDA;
+    if (!make_tmap(&a.tm_wdt, h->WdT, h->Ipad, h->d, h->Ipad, a.bn / 2)) return MLPMOE_ERR_CUDA;
+    a.out_mode = TcLayerArgs::OUT_DIRECT;
+    if (y_dtype == MLPMOE_FP32 && residual == nullptr) a.out_mode = TcLayerArgs::OUT_TMA_STORE;
+    else if (y_dtype == MLPMOE_FP32 && residual == y) a.out_mode = TcLayerArgs::OUT_TMA_ADD;
+    if (a.out_mode != TcLayerArgs::OUT_DIRECT) {
+      if (!make_tmap_t(&a.tm_y, y, h->d, n, h->d, 32, 4)) return MLPMOE_ERR_CUDA;
+    } else {
+      a.tm_y = a.tm_h_st;       // not used by the direct epilogue; any valid map
+    }
+    a.scale = h->scale;
+    a.R = residual;
+    a.Y = y;
+    a.y_bf16 = y_dtype == MLPMOE_BF16;
+    a.n = n; a.d = h->d; a.Ipad = h->Ipad;
+    a.done = h->block_done;
+    a.passed = h->block_done + h->max_blocks;
+    a.status = h->status;
+    const long e0 = rec_event(h, st);
+    CK(launch_tc_layer(a, h->num_sms, st));
+    const long e1 = rec_event(h, st);
+    add_span(h, SPAN_GATEUP, e0, e1);      // the fused kernel is reported in the first slot
+    h->launches += 1;
+    return MLPMOE_OK;
+  }
+  // 65..128 tokens: one CTA per tile, two kernels
   TcGateUpArgs g;
   if (!make_tmap(&g.tm_x, x, h->d, n, h->d, 128)) return MLPMOE_ERR_CUDA;
-  g.tm_w = pair ? h->tm_wgu_pair : h->tm_wgu;
+  g.tm_w = h->tm_wgu;
   g.scale = h->scale;
   g.H = h->ws->H;
   g.n = n; g.d = h->d; g.Ipad = h->Ipad;
   g.status = h->status;
   TcDownArgs dn;
   if (!make_tmap(&dn.tm_h, h->ws->H, h->Ipad, n, h->Ipad, 128)) return MLPMOE_ERR_CUDA;
-  int bn = 128;
-  if (pair) {
-    bn = tc_pair_down_bn(n, h->d, h->num_sms);
-    if (!make_tmap(&dn.tm_w, h->WdT, h->Ipad, h->d, h->Ipad, bn / 2)) return MLPMOE_ERR_CUDA;
-    if (!make_tmap(&g.tm_out, h->ws->H, h->Ipad, n, h->Ipad, 32)) return MLPMOE_ERR_CUDA;
-    if (y_dtype == MLPMOE_FP32) {
-      if (!make_tmap_t(&dn.tm_out, y, h->d, n, h->d, 32, 4)) return MLPMOE_ERR_CUDA;
-    } else {
-      dn.tm_out = dn.tm_h;     // not used by the direct epilogue; any valid map
-    }
-  } else {
-    dn.tm_w = h->tm_wdt;
-  }
+  dn.tm_w = h->tm_wdt;
   dn.R = residual;
   dn.Y = y;
   dn.y_bf16 = y_dtype == MLPMOE_BF16;
   dn.n = n; dn.d = h->d; dn.Ipad = h->Ipad;
   dn.status = h->status;
   const long e0 = rec_event(h, st);
-  CK(pair ? launch_tc_pair_gateup(g, h->num_sms, st) : launch_tc_gateup(g, h->num_sms, st));
+  CK(launch_tc_gateup(g, h->num_sms, st));
   const long e1 = rec_event(h, st);
-  CK(pair ? launch_tc_pair_down(dn, bn, h->num_sms, st) : launch_tc_down(dn, h->num_sms, st));
+  CK(launch_tc_down(dn, h->num_sms, st));
   const long e2 = rec_event(h, st);
   add_span(h, SPAN_GATEUP, e0, e1);
   add_span(h, SPAN_DOWN, e1, e2);
@@ -378,7 +399,7 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
   CK(cudaGetDeviceProperties(&prop, dev));
   if (prop.major != 10) return MLPMOE_ERR_UNSUPPORTED;     // kernels are built for sm_100a only
   CK(tc_gemm_init());
-  CK(tc_pair_init());
+  CK(tc_layer_init());
   CK(decode_init());
 
   mlpmoe_layer_s* h = new (std::nothrow) mlpmoe_layer_s();
@@ -404,6 +425,7 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
   const size_t mat = static_cast<size_t>(d_model) * d_inter * es;
   const int m_blocks = static_cast<int>((d_model + 127) / 128);
   h->max_splits = h->num_sms / m_blocks + 1;
+  h->max_blocks = (max_tokens + 255) / 256;
   h->ws = new (std::nothrow) Workspace();
   bool ok = h->ws != nullptr;
   if (ok) {
@@ -423,6 +445,7 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
        cudaMalloc(&h->fade_work, fade_work_bytes(2 * B)) == cudaSuccess &&
        cudaMalloc(&h->partial, sizeof(float) * static_cast<size_t>(h->max_splits) * d_model * kDecodeMaxTokens) == cudaSuccess &&
        cudaMalloc(&h->counters, sizeof(uint32_t) * m_blocks * 4) == cudaSuccess &&
+       cudaMalloc(&h->block_done, sizeof(uint32_t) * 2 * h->max_blocks) == cudaSuccess &&
        cudaMalloc(&h->status, sizeof(uint32_t)) == cudaSuccess &&
        cudaMalloc(&h->ws->H, static_cast<size_t>(max_tokens) * h->Ipad_max * es) == cudaSuccess &&
        cudaMalloc(&h->ws->xnorm, static_cast<size_t>(max_tokens) * d_model * es) == cudaSuccess &&
@@ -435,6 +458,7 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
   mlpmoe_status_t rc = MLPMOE_OK;
   auto fail = [&](mlpmoe_status_t s) { free_layer(h); return s; };
   if (cudaMemsetAsync(h->counters, 0, sizeof(uint32_t) * m_blocks * 4, st) != cudaSuccess ||
+      cudaMemsetAsync(h->block_done, 0, sizeof(uint32_t) * 2 * h->max_blocks, st) != cudaSuccess ||
       cudaMemsetAsync(h->status, 0, sizeof(uint32_t), st) != cudaSuccess)
     return fail(MLPMOE_ERR_CUDA);
   // canonical copies: one row of d contiguous weights per intermediate neuron, for all three matrices

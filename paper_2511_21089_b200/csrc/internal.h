@@ -79,7 +79,6 @@ cudaError_t launch_simt_down(const float* H, const float* WdT, const float* R, f
 struct TcGateUpArgs {
   CUtensorMap tm_x;     // X   [n x d]            bf16, box 64 x 128, 128B swizzle
   CUtensorMap tm_w;     // Wgu [2*Ipad x d]       bf16, box 64 x 256
-  CUtensorMap tm_out;   // H   [n x Ipad]         bf16, box 64 x 32 (CTA-pair kernel's TMA-store epilogue)
   const float* scale;   // [Ipad]
   void* H;              // [n x Ipad] bf16
   int64_t n, d, Ipad;
@@ -88,7 +87,6 @@ struct TcGateUpArgs {
 struct TcDownArgs {
   CUtensorMap tm_h;     // H   [n x Ipad]         bf16, box 64 x 128
   CUtensorMap tm_w;     // WdT [d x Ipad]         bf16, box 64 x 128
-  CUtensorMap tm_out;   // Y   [n x d]            fp32, box 32 x 32 (CTA-pair kernel's TMA-store epilogue)
   const float* R;       // optional fp32 residual [n x d]
   void* Y;              // [n x d] fp32 or bf16
   int y_bf16;
@@ -99,13 +97,28 @@ cudaError_t launch_tc_gateup(const TcGateUpArgs& a, int num_sms, cudaStream_t st
 cudaError_t launch_tc_down(const TcDownArgs& a, int num_sms, cudaStream_t st);
 cudaError_t tc_gemm_init();   // opt in to the large dynamic shared memory sizes (once per process)
 
-// -------------------------------------------------------------- tc_gemm2.cu --
-// CTA-pair (cta_group::2) versions: tm_w of the gate|up call has box 64 x 128, tm_w of the down
-// call has box 64 x bn/2 (each CTA of a pair stages half of the weight rows of a tile).
-cudaError_t tc_pair_init();
-int tc_pair_down_bn(int64_t n, int64_t d, int num_sms);
-cudaError_t launch_tc_pair_gateup(const TcGateUpArgs& a, int num_sms, cudaStream_t st);
-cudaError_t launch_tc_pair_down(const TcDownArgs& a, int bn, int num_sms, cudaStream_t st);
+// -------------------------------------------------------------- tc_layer.cu --
+// Both GEMMs of a layer call in one persistent CTA-pair kernel (n > 128).
+struct TcLayerArgs {
+  enum { OUT_DIRECT = 0, OUT_TMA_STORE = 1, OUT_TMA_ADD = 2 };   // how the down epilogue leaves
+  CUtensorMap tm_x;      // X   [n x d]       bf16, box 64 x 128
+  CUtensorMap tm_wgu;    // Wgu [2 Ipad x d]  bf16, box 64 x 128
+  CUtensorMap tm_h_st;   // H   [n x Ipad]    bf16, box 64 x 32
+  CUtensorMap tm_h_ld;   // H   [n x Ipad]    bf16, box 64 x 128
+  CUtensorMap tm_wdt;    // WdT [d x Ipad]    bf16, box 64 x bn/2
+  CUtensorMap tm_y;      // Y   [n x d]       fp32, box 32 x 32 (unused by OUT_DIRECT)
+  const float* scale;
+  const float* R;
+  void* Y;
+  int y_bf16, out_mode, bn;
+  int64_t n, d, Ipad;
+  uint32_t* done;        // [ceil(n / 256)] zero between calls
+  uint32_t* passed;      // [ceil(n / 256)] zero between calls
+  uint32_t* status;
+};
+cudaError_t tc_layer_init();
+int tc_layer_down_bn(int64_t n, int64_t d, int num_sms);
+cudaError_t launch_tc_layer(const TcLayerArgs& a, int num_sms, cudaStream_t st);
 
 // ---------------------------------------------------------------- decode.cu --
 struct DecodeArgs {
