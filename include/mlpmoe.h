@@ -264,6 +264,18 @@ mlpmoe_status_t mlpmoe_host_schedule(int32_t B, const int64_t* d_b, const float*
                                      int64_t* seg_start, int64_t* seg_len, int32_t* n_segs,
                                      int64_t* n_active);
 
+/*
+ * The static tile schedule of the fused prefill kernel for n_tokens tokens: which CTA pair runs
+ * which gate|up / down tiles in which order (set-up logic, no CUDA call).  Down tiles are cut into
+ * ksplit (1..4) slices of the contraction range.  tiles: capacity
+ * ceil(n/256) * (n_active_pad/128 + ksplit * ceil(d_model/bn)); offsets: capacity num_sms/2 + 1.
+ * Tile code: bit 31 = down tile, bits 16..30 = column-tile index (down: column tile * ksplit +
+ * slice), bits 0..15 = 256-token block.
+ */
+mlpmoe_status_t mlpmoe_host_tile_schedule(int64_t n_tokens, int64_t d_model, int64_t n_active_pad, int32_t bn,
+                                          int32_t ksplit, int32_t num_sms, int32_t* tiles, int32_t* n_tiles,
+                                          int32_t* offsets);
+
 #ifdef __cplusplus
 }
 #endif

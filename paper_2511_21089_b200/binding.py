@@ -61,6 +61,8 @@ SIGNATURES = {
     "mlpmoe_host_fade_position": (c_int32, [c_double, c_int64, POINTER(c_int64)]),
     "mlpmoe_host_fade_position_default": (c_int32, [c_int32, c_int32, c_int64, POINTER(c_int64)]),
     "mlpmoe_host_prune_alpha": (c_int32, [c_int32, POINTER(c_float), POINTER(c_uint8), c_int32, POINTER(c_float)]),
+    "mlpmoe_host_tile_schedule": (c_int32, [c_int64, c_int64, c_int64, c_int32, c_int32, c_int32, POINTER(c_int32), POINTER(c_int32),
+                                            POINTER(c_int32)]),
     "mlpmoe_host_schedule": (c_int32, [c_int32, POINTER(c_int64), POINTER(c_float), POINTER(c_uint8), POINTER(c_int32),
                                        POINTER(c_int32), POINTER(c_int64), POINTER(c_int64), POINTER(c_int32),
                                        POINTER(c_int64)]),
@@ -275,3 +277,17 @@ def mlpmoe_host_schedule(d_b: Sequence[int], alpha_eff: Sequence[float], live=No
     _check(lib.mlpmoe_host_schedule(B, _arr(d_b, c_int64), _arr(alpha_eff, c_float), live_arr, br, ctypes.byref(nb), ss, sl,
                                     ctypes.byref(ns), ctypes.byref(na)), "mlpmoe_host_schedule")
     return list(br[:nb.value]), [(ss[i], sl[i]) for i in range(ns.value)], na.value
+
+
+def mlpmoe_host_tile_schedule(n_tokens: int, d_model: int, n_active_pad: int, bn: int, ksplit: int = 1, num_sms: int = 148):
+    """Returns one list of (is_down, column_tile [* ksplit + slice], token_block) per CTA pair."""
+    cap = ((n_tokens + 255) // 256) * (n_active_pad // 128 + ksplit * ((d_model + bn - 1) // bn))
+    tiles = (c_int32 * cap)()
+    n_tiles = c_int32()
+    offs = (c_int32 * (num_sms // 2 + 1))()
+    _check(lib.mlpmoe_host_tile_schedule(n_tokens, d_model, n_active_pad, bn, ksplit, num_sms, tiles, ctypes.byref(n_tiles), offs),
+           "mlpmoe_host_tile_schedule")
+    out = []
+    for c in range(num_sms // 2):
+        out.append([((t >> 31) & 1, (t >> 16) & 0x7FFF, t & 0xFFFF) for t in tiles[offs[c]:offs[c + 1]]])
+    return out

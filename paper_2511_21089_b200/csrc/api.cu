@@ -174,6 +174,10 @@ struct mlpmoe_layer_s {
   uint32_t* counters = nullptr;
   uint32_t* block_done = nullptr;                           // [2 x ceil(max_tokens / 256)] gate|up completion counters
   int64_t max_blocks = 0;
+  int32_t* tile_sched = nullptr;                            // device: tile sequences + offsets of the fused prefill kernel
+  int64_t sched_capacity = 0, sched_n = -1, sched_Ipad = -1;
+  int sched_bn = 0, sched_ksplit = 0, sched_tiles = 0;
+  std::vector<int32_t> sched_host;
   int max_splits = 1;
   uint32_t* status = nullptr;
   int64_t launches = 0;
@@ -208,7 +212,7 @@ void free_layer(mlpmoe_layer_s* h) {
   cudaFree(h->Wg_c); cudaFree(h->Wu_c); cudaFree(h->Wd_c);
   cudaFree(h->Wgu); cudaFree(h->WdT);
   cudaFree(h->scale); cudaFree(h->src_row); cudaFree(h->row_nnz);
-  cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->block_done); cudaFree(h->status);
+  cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->block_done); cudaFree(h->tile_sched); cudaFree(h->status);
   ws_release(h->ws);
   delete h;
 }
@@ -328,6 +332,20 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
     a.Y = y;
     a.y_bf16 = y_dtype == MLPMOE_BF16;
     a.n = n; a.d = h->d; a.Ipad = h->Ipad;
+    a.ksplit = tc_layer_ksplit(n, h->d, h->Ipad, a.bn, a.out_mode, h->num_sms);
+    if (h->sched_n != n || h->sched_Ipad != h->Ipad || h->sched_bn != a.bn || h->sched_ksplit != a.ksplit) {
+      // first call with this token count since the last reschedule: build and upload the tile sequences
+      std::vector<int32_t> tiles, offs;
+      tc_layer_schedule(n, h->d, h->Ipad, a.bn, a.ksplit, h->num_sms, &tiles, &offs);
+      if (static_cast<int64_t>(tiles.size() + offs.size()) > h->sched_capacity) return MLPMOE_ERR_UNSUPPORTED;
+      h->sched_host = tiles;
+      h->sched_host.insert(h->sched_host.end(), offs.begin(), offs.end());
+      h->sched_tiles = static_cast<int>(tiles.size());
+      CK(cudaMemcpyAsync(h->tile_sched, h->sched_host.data(), sizeof(int32_t) * h->sched_host.size(), cudaMemcpyHostToDevice, st));
+      h->sched_n = n; h->sched_Ipad = h->Ipad; h->sched_bn = a.bn; h->sched_ksplit = a.ksplit;
+    }
+    a.tile_list = h->tile_sched;
+    a.list_offsets = h->tile_sched + h->sched_tiles;
     a.done = h->block_done;
     a.passed = h->block_done + h->max_blocks;
     a.status = h->status;
@@ -426,6 +444,7 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
   const int m_blocks = static_cast<int>((d_model + 127) / 128);
   h->max_splits = h->num_sms / m_blocks + 1;
   h->max_blocks = (max_tokens + 255) / 256;
+  h->sched_capacity = h->max_blocks * (h->Ipad_max / 128 + 4 * ((d_model + 63) / 64)) + h->num_sms / 2 + 2;
   h->ws = new (std::nothrow) Workspace();
   bool ok = h->ws != nullptr;
   if (ok) {
@@ -446,6 +465,7 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
        cudaMalloc(&h->partial, sizeof(float) * static_cast<size_t>(h->max_splits) * d_model * kDecodeMaxTokens) == cudaSuccess &&
        cudaMalloc(&h->counters, sizeof(uint32_t) * m_blocks * 4) == cudaSuccess &&
        cudaMalloc(&h->block_done, sizeof(uint32_t) * 2 * h->max_blocks) == cudaSuccess &&
+       cudaMalloc(&h->tile_sched, sizeof(int32_t) * h->sched_capacity) == cudaSuccess &&
        cudaMalloc(&h->status, sizeof(uint32_t)) == cudaSuccess &&
        cudaMalloc(&h->ws->H, static_cast<size_t>(max_tokens) * h->Ipad_max * es) == cudaSuccess &&
        cudaMalloc(&h->ws->xnorm, static_cast<size_t>(max_tokens) * d_model * es) == cudaSuccess &&
@@ -754,6 +774,20 @@ mlpmoe_status_t mlpmoe_host_schedule(int32_t B, const int64_t* d_b, const float*
   if (n_segs) *n_segs = static_cast<int32_t>(s.seg_start.size());
   if (n_active) *n_active = s.n_active;
   (void)I;
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_host_tile_schedule(int64_t n_tokens, int64_t d_model, int64_t n_active_pad, int32_t bn,
+                                          int32_t ksplit, int32_t num_sms, int32_t* tiles, int32_t* n_tiles,
+                                          int32_t* offsets) {
+  if (n_tokens <= 0 || d_model <= 0 || n_active_pad <= 0 || n_active_pad % 128 != 0 || bn < 32 || bn > 256 || bn % 32 != 0 ||
+      num_sms < 2 || ksplit < 1 || ksplit > 4 || !tiles || !n_tiles || !offsets)
+    return MLPMOE_ERR_INVALID_ARG;
+  std::vector<int32_t> t, o;
+  tc_layer_schedule(n_tokens, d_model, n_active_pad, bn, ksplit, num_sms, &t, &o);
+  std::memcpy(tiles, t.data(), sizeof(int32_t) * t.size());
+  std::memcpy(offsets, o.data(), sizeof(int32_t) * o.size());
+  *n_tiles = static_cast<int32_t>(t.size());
   return MLPMOE_OK;
 }
 

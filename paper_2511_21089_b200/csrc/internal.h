@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include <utility>
+#include <vector>
 
 namespace mlpmoe {
 
@@ -110,14 +111,19 @@ struct TcLayerArgs {
   const float* scale;
   const float* R;
   void* Y;
-  int y_bf16, out_mode, bn;
+  int y_bf16, out_mode, bn, ksplit;
   int64_t n, d, Ipad;
+  const int32_t* tile_list;     // device: per-pair tile sequences from tc_layer_schedule
+  const int32_t* list_offsets;  // device: [num_sms / 2 + 1]
   uint32_t* done;        // [ceil(n / 256)] zero between calls
   uint32_t* passed;      // [ceil(n / 256)] zero between calls
   uint32_t* status;
 };
 cudaError_t tc_layer_init();
 int tc_layer_down_bn(int64_t n, int64_t d, int num_sms);
+int tc_layer_ksplit(int64_t n, int64_t d, int64_t Ipad, int bn, int out_mode, int num_sms);
+int64_t tc_layer_schedule(int64_t n, int64_t d, int64_t Ipad, int bn, int ksplit, int num_sms, std::vector<int32_t>* tiles,
+                          std::vector<int32_t>* offsets);
 cudaError_t launch_tc_layer(const TcLayerArgs& a, int num_sms, cudaStream_t st);
 
 // ---------------------------------------------------------------- decode.cu --

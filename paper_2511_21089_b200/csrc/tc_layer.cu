@@ -24,6 +24,9 @@
 // memory and TMA stores).  Barriers: "empty" and "accumulator full" per CTA, reached by
 // multicast commits; "full" and "accumulator empty" live in the even CTA and are signalled from
 // both.  No load uses cluster multicast.  Every wait is bounded.
+#include <utility>
+#include <vector>
+
 #include "tc_common.cuh"
 
 namespace mlpmoe {
@@ -55,22 +58,28 @@ struct LayerParams {
   int m_pairs;            // 256-token blocks
   int n1, kb1;            // gate|up: tiles per token block (Ipad / 128), K-steps (d / 64)
   int n2, kb2, bn;        // down: tiles per token block, K-steps (Ipad / 64), tile width
+  int ksplit;             // down tiles are cut into this many K slices (> 1 only when Y is accumulated into)
+  const int32_t* tile_list;     // per-cluster tile sequences, concatenated (see encode_tile)
+  const int32_t* list_offsets;  // [clusters + 1] start of each cluster's sequence
   uint32_t* done;         // [m_pairs] finished gate|up tile arrivals; zero between calls
   uint32_t* passed;       // [m_pairs] down-tile producers that have seen the block complete; zero between calls
   uint32_t* status;
 };
 
 struct Tile {
-  int is_down, m_pair, n_blk;
+  int is_down, m_pair, n_blk, kslice;
 };
 
-__device__ __forceinline__ Tile decode_tile(int tile, const LayerParams& p) {
+// Tile code: bit 31 = down tile, bits 16..30 = tile index along the output columns, bits 0..15 =
+// 256-token block.
+// For down tiles the column field holds column_tile * ksplit + K slice.
+__device__ __forceinline__ Tile decode_tile(int32_t code, int ksplit) {
   Tile t;
-  const int t1 = p.m_pairs * p.n1;
-  t.is_down = tile >= t1;
-  const int idx = t.is_down ? tile - t1 : tile;
-  t.m_pair = idx % p.m_pairs;          // token block fastest: concurrently running tiles share weight tiles
-  t.n_blk = idx / p.m_pairs;
+  t.is_down = (static_cast<uint32_t>(code) >> 31) & 1;
+  const int col = (code >> 16) & 0x7FFF;
+  t.n_blk = t.is_down ? col / ksplit : col;
+  t.kslice = t.is_down ? col % ksplit : 0;
+  t.m_pair = code & 0xFFFF;
   return t;
 }
 
@@ -142,9 +151,9 @@ tc_layer_kernel(const __grid_constant__ CUtensorMap tm_x,        // X   [n x d] 
   const uint32_t tmem_base = *tmem_slot;
   griddep_launch_dependents();          // the next kernel may begin its set-up
   griddep_wait();                       // inputs written by earlier kernels are complete and visible
-  const int num_tiles = p.m_pairs * (p.n1 + p.n2);
-  const int first_tile = static_cast<int>(cluster_id_x());
-  const int tile_step = static_cast<int>(cluster_count_x());
+  // this CTA pair's tile sequence (the same for every role of both CTAs)
+  const int list_begin = p.list_offsets[cluster_id_x()];
+  const int list_end = p.list_offsets[cluster_id_x() + 1];
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -156,11 +165,12 @@ tc_layer_kernel(const __grid_constant__ CUtensorMap tm_x,        // X   [n x d] 
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
-        const Tile t = decode_tile(tile, p);
+      for (int i = list_begin; ok && i < list_end; ++i) {
+        const Tile t = decode_tile(p.tile_list[i], p.ksplit);
         const int bn = t.is_down ? p.bn : 256;
         const int half_rows = bn / 2;
-        const int kbs = t.is_down ? p.kb2 : p.kb1;
+        const int kb_lo = t.is_down ? t.kslice * p.kb2 / p.ksplit : 0;
+        const int kb_hi = t.is_down ? (t.kslice + 1) * p.kb2 / p.ksplit : p.kb1;
         const CUtensorMap* ma = t.is_down ? &tm_h_ld : &tm_x;
         const CUtensorMap* mb = t.is_down ? &tm_wdt : &tm_wgu;
         const int row_a = (t.m_pair * 2 + static_cast<int>(rank)) * BM;
@@ -170,13 +180,13 @@ tc_layer_kernel(const __grid_constant__ CUtensorMap tm_x,        // X   [n x d] 
           // H rows of this token block are complete once every gate|up tile of the block has arrived
           if (!wait_count(p.done + t.m_pair, static_cast<uint32_t>(p.n1) * ARRIVALS_PER_GATEUP_TILE, abort_flag)) { ok = false; break; }
           fence_proxy_async_all();       // the TMA loads below must observe what that acquire made visible
-          // the last of the 2 * n2 producers of this block to get here re-arms the counters for the next call
-          if (atomicAdd(p.passed + t.m_pair, 1u) == static_cast<uint32_t>(2 * p.n2 - 1)) {
+          // the last of the 2 * n2 * ksplit producers of this block to get here re-arms the counters for the next call
+          if (atomicAdd(p.passed + t.m_pair, 1u) == static_cast<uint32_t>(2 * p.n2 * p.ksplit - 1)) {
             p.done[t.m_pair] = 0;
             p.passed[t.m_pair] = 0;
           }
         }
-        for (int kb = 0; kb < kbs; ++kb) {
+        for (int kb = kb_lo; kb < kb_hi; ++kb) {
           if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, WAIT_NS)) { ok = false; break; }
           uint8_t* sa = smem + stage * STAGE_BYTES;
           const uint32_t full_even = map_to_cta(smem_u32(&full_bar[stage]), 0);
@@ -198,14 +208,15 @@ tc_layer_kernel(const __grid_constant__ CUtensorMap tm_x,        // X   [n x d] 
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
-        const Tile t = decode_tile(tile, p);
-        const int kbs = t.is_down ? p.kb2 : p.kb1;
+      for (int i = list_begin; ok && i < list_end; ++i) {
+        const Tile t = decode_tile(p.tile_list[i], p.ksplit);
+        const int kb_lo = t.is_down ? t.kslice * p.kb2 / p.ksplit : 0;
+        const int kb_hi = t.is_down ? (t.kslice + 1) * p.kb2 / p.ksplit : p.kb1;
         const uint32_t idesc = make_idesc_bf16_f32(256, static_cast<uint32_t>(t.is_down ? p.bn : 256));
         if (!mbar_wait_bounded(&tempty_bar[acc], acc_phase ^ 1u, abort_flag, WAIT_NS)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * ACC_STRIDE);
-        for (int kb = 0; kb < kbs; ++kb) {
+        for (int kb = kb_lo; kb < kb_hi; ++kb) {
           if (!mbar_wait_bounded(&full_bar[stage], phase, abort_flag, WAIT_NS)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES);
@@ -213,7 +224,7 @@ tc_layer_kernel(const __grid_constant__ CUtensorMap tm_x,        // X   [n x d] 
           const uint64_t b_desc = make_desc_sw128_kmajor(sa + A_BYTES);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k)
-            umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb > kb_lo || k > 0) ? 1u : 0u);
           umma_commit_pair(&empty_bar[stage], 3);      // frees this stage in both CTAs
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -241,8 +252,8 @@ tc_layer_kernel(const __grid_constant__ CUtensorMap tm_x,        // X   [n x d] 
     ep.cols = p.d;
     ep.ld = p.d;
     ep.out_bf16 = p.y_bf16;
-    for (int tile = first_tile; tile < num_tiles; tile += tile_step) {
-      const Tile t = decode_tile(tile, p);
+    for (int i = list_begin; i < list_end; ++i) {
+      const Tile t = decode_tile(p.tile_list[i], p.ksplit);
       bool ok = mbar_wait_bounded(&tfull_bar[acc], acc_phase, abort_flag, WAIT_NS);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
@@ -314,6 +325,136 @@ int tc_layer_down_bn(int64_t n, int64_t d, int num_sms) {
   return best;
 }
 
+namespace {
+inline int32_t encode_tile(bool is_down, int n_blk, int m_pair) {
+  return static_cast<int32_t>((is_down ? 0x80000000u : 0u) | (static_cast<uint32_t>(n_blk) << 16) | static_cast<uint32_t>(m_pair));
+}
+// Estimated cycles of one K-step of a 256 x bn pair tile: tensor-core time or L2 fill time.
+inline int64_t kstep_cycles(int bn) {
+  const int64_t mma = 2 * bn, fill = (A_BYTES + (bn / 2) * BK * 2) / 50;
+  return mma > fill ? mma : fill;
+}
+}  // namespace
+
+// Static tile schedule: which CTA pair runs which tiles, in which order.  A greedy list scheduler
+// over estimated tile costs.  Token blocks are taken in groups; a group's gate|up tiles run with
+// the token block fastest (tiles in flight share weight tiles, the group shares one pass over the
+// weights), and its down tiles become eligible once the simulation has finished every gate|up
+// tile of their token block, so that they are handed to pairs that would otherwise idle at the end
+// of a wave.  Every pair's sequence follows one global order in which a down tile comes after all
+// gate|up tiles of its token block: the waits inside the kernel therefore cannot form a cycle.
+int64_t tc_layer_schedule(int64_t n, int64_t d, int64_t Ipad, int bn, int ksplit, int num_sms, std::vector<int32_t>* tiles,
+                          std::vector<int32_t>* offsets) {
+  const int pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
+  const int m_pairs = static_cast<int>((n + 255) / 256);
+  const int n1 = static_cast<int>(Ipad / 128), n2 = static_cast<int>((d + bn - 1) / bn) * ksplit;   // down items per token block
+  const int64_t cost_g = ((d + BK - 1) / BK) * kstep_cycles(256) + 1500;
+  const int64_t cost_d = (Ipad / BK) * kstep_cycles(bn) / ksplit + 1500 + 24 * bn;     // + exposed part of the epilogue
+  // Group size.  At least enough token blocks to keep every pair busy on one pass over the weight
+  // tiles.  Weights that fit in L2 need no more (small groups finish their token blocks early, so
+  // down tiles become eligible early); larger weights are streamed from HBM once per group, so
+  // take at least 8 token blocks per pass.
+  int group = (pairs + n1 - 1) / n1 + 1;
+  const bool weights_fit_l2 = 3 * d * Ipad * 2 <= (int64_t(48) << 20);
+  if (!weights_fit_l2 && group < 8) group = 8;
+  if (group > m_pairs) group = m_pairs;
+  std::vector<int32_t> g_order;
+  g_order.reserve(static_cast<size_t>(m_pairs) * n1);
+  for (int g0 = 0; g0 < m_pairs; g0 += group)
+    for (int nb = 0; nb < n1; ++nb)
+      for (int m = g0; m < g0 + group && m < m_pairs; ++m) g_order.push_back(encode_tile(false, nb, m));
+  std::vector<int64_t> avail(pairs, 0);
+  std::vector<std::vector<int32_t>> lists(pairs);
+  std::vector<int> g_left(m_pairs, n1);
+  std::vector<int64_t> block_done_at(m_pairs, 0);
+  struct Ready { int64_t at; int32_t code; };
+  std::vector<Ready> d_ready;          // FIFO of eligible down tiles
+  size_t d_head = 0, g_next = 0;
+  const size_t total = static_cast<size_t>(m_pairs) * (n1 + n2);
+  size_t assigned = 0;
+  // down tiles are the large items: no pair takes more than its share of them while gate|up tiles remain
+  const int d_quota = static_cast<int>((static_cast<int64_t>(m_pairs) * n2 + pairs - 1) / pairs);
+  std::vector<int> d_taken(pairs, 0);
+  // pending completions of simulated gate|up tiles: (finish time, token block)
+  std::vector<std::pair<int64_t, int>> running;
+  auto retire = [&](int64_t now) {
+    for (size_t i = 0; i < running.size();) {
+      if (running[i].first <= now) {
+        const int m = running[i].second;
+        if (block_done_at[m] < running[i].first) block_done_at[m] = running[i].first;
+        if (--g_left[m] == 0)
+          for (int nb = 0; nb < n2; ++nb) d_ready.push_back({block_done_at[m], encode_tile(true, nb, m)});
+        running[i] = running.back();
+        running.pop_back();
+      } else {
+        ++i;
+      }
+    }
+  };
+  while (assigned < total) {
+    int c = 0;
+    for (int i = 1; i < pairs; ++i)
+      if (avail[i] < avail[c]) c = i;
+    int64_t now = avail[c];
+    retire(now);
+    int cd = -1;                         // the earliest-free pair that still has room for a down tile
+    if (d_head < d_ready.size()) {
+      for (int i = 0; i < pairs; ++i)
+        if (d_taken[i] < d_quota && (cd < 0 || avail[i] < avail[cd])) cd = i;
+      if (cd < 0 && g_next >= g_order.size()) cd = c;    // everyone has a share and nothing else is left
+    }
+    if (cd >= 0) {
+      ++d_taken[cd];
+      lists[cd].push_back(d_ready[d_head].code);
+      const int64_t t0 = avail[cd] > d_ready[d_head].at ? avail[cd] : d_ready[d_head].at;
+      avail[cd] = t0 + cost_d;
+      ++d_head;
+    } else if (g_next < g_order.size()) {
+      const int32_t code = g_order[g_next++];
+      lists[c].push_back(code);
+      avail[c] = now + cost_g;
+      running.push_back({avail[c], static_cast<int>(code & 0xFFFF)});
+    } else {
+      // only down tiles whose gate|up tiles are still running in the simulation remain: advance time
+      int64_t next = -1;
+      for (const auto& r : running)
+        if (next < 0 || r.first < next) next = r.first;
+      avail[c] = next > now ? next : now + 1;
+      continue;
+    }
+    ++assigned;
+  }
+  tiles->clear();
+  offsets->assign(1, 0);
+  for (int c = 0; c < pairs; ++c) {
+    tiles->insert(tiles->end(), lists[c].begin(), lists[c].end());
+    offsets->push_back(static_cast<int32_t>(tiles->size()));
+  }
+  int64_t makespan = 0;                 // simulated finish time of the last pair, in cycles of the cost model
+  for (int c = 0; c < pairs; ++c) makespan = avail[c] > makespan ? avail[c] : makespan;
+  return makespan;
+}
+
+// Number of K slices per down tile (1..4): the one whose simulated schedule finishes first.
+// Slicing is only possible when Y is accumulated into (each slice adds its part), and only matters
+// when a CTA pair gets few tiles: whole down tiles, several times longer than gate|up tiles, then
+// cannot be balanced across the pairs.
+int tc_layer_ksplit(int64_t n, int64_t d, int64_t Ipad, int bn, int out_mode, int num_sms) {
+  if (out_mode != TcLayerArgs::OUT_TMA_ADD) return 1;
+  const int64_t pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
+  const int64_t m_pairs = (n + 255) / 256;
+  if (m_pairs * (Ipad / 128 + (d + bn - 1) / bn) >= 24 * pairs) return 1;
+  int best = 1;
+  int64_t best_t = -1;
+  std::vector<int32_t> t, o;
+  for (int k = 1; k <= 4; ++k) {
+    if (k > 1 && (Ipad / BK) / k < 8) break;
+    const int64_t span = tc_layer_schedule(n, d, Ipad, bn, k, num_sms, &t, &o);
+    if (best_t < 0 || span < best_t - best_t / 50) { best = k; best_t = span; }   // a finer cut must win by 2 %
+  }
+  return best;
+}
+
 cudaError_t launch_tc_layer(const TcLayerArgs& a, int num_sms, cudaStream_t st) {
   if (a.n == 0) return cudaSuccess;
   LayerParams p{};
@@ -330,11 +471,13 @@ cudaError_t launch_tc_layer(const TcLayerArgs& a, int num_sms, cudaStream_t st) 
   p.bn = a.bn;
   p.n2 = static_cast<int>((a.d + a.bn - 1) / a.bn);
   p.kb2 = static_cast<int>(a.Ipad / BK);
+  p.ksplit = a.ksplit;
+  p.tile_list = a.tile_list;
+  p.list_offsets = a.list_offsets;
   p.done = a.done;
   p.passed = a.passed;
   p.status = a.status;
-  const int tiles = p.m_pairs * (p.n1 + p.n2);
-  const int pairs = tiles < num_sms / 2 ? tiles : num_sms / 2;
+  const int pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;     // pairs without tiles have empty sequences
   return launch_pdl(tc_layer_kernel, dim3(2 * pairs), dim3(NUM_THREADS), SMEM_BYTES, st, a.tm_x, a.tm_wgu, a.tm_h_st, a.tm_h_ld,
                     a.tm_wdt, a.tm_y, p);
 }

@@ -136,3 +136,48 @@ def test_synth_generators():
     assert sum(k) == 12 and k == synth.keep_set((7,), 16, 4)
     assert [synth.n_drop_for_ratio(B, r) for B in (4, 32, 128) for r in (0.0, 0.1, 0.2, 0.4)] == \
         [0, 0, 1, 2, 0, 3, 6, 13, 0, 13, 26, 51]
+
+
+@pytest.mark.parametrize("n,d,Ipad,bn,ks", [(4096, 896, 3712, 224, 1), (4096, 896, 3712, 224, 3), (300, 320, 512, 128, 4),
+                                            (8192, 4096, 14336, 256, 1), (2048, 4096, 11520, 256, 2),
+                                            (16384, 4096, 14336, 256, 1), (129, 64, 128, 64, 1)])
+def test_tile_schedule_is_complete_and_cannot_deadlock(lib, n, d, Ipad, bn, ks):
+    """Every tile exactly once; and whatever the tiles' real durations turn out to be, running the
+    per-pair sequences with 'a down tile waits for all gate|up tiles of its token block' finishes."""
+    lists = lib.mlpmoe_host_tile_schedule(n, d, Ipad, bn, ks, 148)
+    m_pairs, n1, n2 = (n + 255) // 256, Ipad // 128, ks * ((d + bn - 1) // bn)
+    flat = [t for l in lists for t in l]
+    assert len(flat) == len(set(flat)) == m_pairs * (n1 + n2)
+    assert set(flat) == {(0, nb, m) for nb in range(n1) for m in range(m_pairs)} | {(1, nb, m) for nb in range(n2) for m in range(m_pairs)}
+    rng = np.random.default_rng(n)
+    for trial in range(3):
+        dur = {t: float(rng.uniform(0.1, 10.0)) for t in flat}            # arbitrary durations
+        pos = [0] * len(lists)
+        clock = [0.0] * len(lists)
+        left = {m: n1 for m in range(m_pairs)}
+        done_at = {m: 0.0 for m in range(m_pairs)}
+        remaining = len(flat)
+        while remaining:
+            progressed = False
+            # run the pair with the smallest clock whose next tile is runnable
+            order = sorted(range(len(lists)), key=lambda c: clock[c])
+            for c in order:
+                if pos[c] >= len(lists[c]):
+                    continue
+                t = lists[c][pos[c]]
+                if t[0] == 1 and left[t[2]] > 0:
+                    continue                                           # blocked: its token block is not complete
+                start = max(clock[c], done_at[t[2]]) if t[0] == 1 else clock[c]
+                clock[c] = start + dur[t]
+                if t[0] == 0:
+                    left[t[2]] -= 1
+                    done_at[t[2]] = max(done_at[t[2]], clock[c])
+                pos[c] += 1
+                remaining -= 1
+                progressed = True
+                break
+            assert progressed, "every pair is blocked on a down tile: the schedule can deadlock"
+    # balance under the cost model: no pair gets more than its share plus one large tile
+    loads = [sum((Ipad // 64) * max(2 * bn, (16384 + bn * 64) // 50) // ks if t[0] else ((d + 63) // 64) * 655 for t in l) for l in lists]
+    if m_pairs * (n1 + n2) >= 4 * 74:
+        assert max(loads) <= 1.35 * (sum(loads) / len(loads))
