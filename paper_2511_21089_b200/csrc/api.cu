@@ -176,7 +176,7 @@ struct mlpmoe_layer_s {
   int64_t max_blocks = 0;
   int32_t* tile_sched = nullptr;                            // device: tile sequences + offsets of the fused prefill kernel
   int64_t sched_capacity = 0, sched_n = -1, sched_Ipad = -1;
-  int sched_bn = 0, sched_ksplit = 0, sched_tiles = 0;
+  int sched_bn = 0, sched_ksplit = 0, sched_tiles = 0, sched_out_mode = -1;
   std::vector<int32_t> sched_host;
   int max_splits = 1;
   uint32_t* status = nullptr;
@@ -332,18 +332,20 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
     a.Y = y;
     a.y_bf16 = y_dtype == MLPMOE_BF16;
     a.n = n; a.d = h->d; a.Ipad = h->Ipad;
-    a.ksplit = tc_layer_ksplit(n, h->d, h->Ipad, a.bn, a.out_mode, h->num_sms);
-    if (h->sched_n != n || h->sched_Ipad != h->Ipad || h->sched_bn != a.bn || h->sched_ksplit != a.ksplit) {
-      // first call with this token count since the last reschedule: build and upload the tile sequences
+    if (h->sched_n != n || h->sched_Ipad != h->Ipad || h->sched_bn != a.bn || h->sched_out_mode != a.out_mode) {
+      // first call with this token count / output mode since the last reschedule: choose the K
+      // slicing, build the tile sequences (host work) and upload them
+      const int ksplit = tc_layer_ksplit(n, h->d, h->Ipad, a.bn, a.out_mode, h->num_sms);
       std::vector<int32_t> tiles, offs;
-      tc_layer_schedule(n, h->d, h->Ipad, a.bn, a.ksplit, h->num_sms, &tiles, &offs);
+      tc_layer_schedule(n, h->d, h->Ipad, a.bn, ksplit, h->num_sms, &tiles, &offs);
       if (static_cast<int64_t>(tiles.size() + offs.size()) > h->sched_capacity) return MLPMOE_ERR_UNSUPPORTED;
       h->sched_host = tiles;
       h->sched_host.insert(h->sched_host.end(), offs.begin(), offs.end());
       h->sched_tiles = static_cast<int>(tiles.size());
       CK(cudaMemcpyAsync(h->tile_sched, h->sched_host.data(), sizeof(int32_t) * h->sched_host.size(), cudaMemcpyHostToDevice, st));
-      h->sched_n = n; h->sched_Ipad = h->Ipad; h->sched_bn = a.bn; h->sched_ksplit = a.ksplit;
+      h->sched_n = n; h->sched_Ipad = h->Ipad; h->sched_bn = a.bn; h->sched_ksplit = ksplit; h->sched_out_mode = a.out_mode;
     }
+    a.ksplit = h->sched_ksplit;
     a.tile_list = h->tile_sched;
     a.list_offsets = h->tile_sched + h->sched_tiles;
     a.done = h->block_done;
