@@ -66,3 +66,17 @@ class Case:
         h = lib.mlpmoe_create(self.d, self.I, self.d_b, wg, wu, wd, self.alpha, dtype, layout, max_tokens, stream_ptr())
         torch.cuda.synchronize()
         return h
+
+
+def layer_rms(inputs, out):
+    """RMS of every layer's own contribution y_l = x_{l+1} - x_l in the oracle's run."""
+    xs = list(inputs) + [out]
+    return [float(np.sqrt(np.mean((xs[l + 1] - xs[l]) ** 2))) for l in range(len(inputs))]
+
+
+def stack_tolerance(inputs, out):
+    """End-to-end bound for a deep stack, as a multiple of RMS(output): every layer's contribution
+    may be off by TOL_BF16 * RMS(y_l); the stack output is the sum of the contributions, so to first
+    order its error is bounded by the sum of those, and the later layers' response to the perturbed
+    stream (damped by RMSNorm, since the stream's RMS grows with depth) is allowed the same again."""
+    return 2.0 * TOL_BF16 * sum(layer_rms(inputs, out)) / float(np.sqrt(np.mean(out ** 2)))

@@ -14,7 +14,7 @@ import torch
 
 import oracle
 from paper_2511_21089_b200 import synth
-from tests.helpers import TOL_BF16, bits_of, dev_bf16, dev_f32, rel_err, stream_ptr
+from tests.helpers import TOL_BF16, bits_of, dev_bf16, dev_f32, rel_err, stack_tolerance, stream_ptr
 
 pytestmark = pytest.mark.gpu
 
@@ -97,12 +97,6 @@ def make_handles(lib, dev, d_b, max_tokens, prune=None):
     return handles
 
 
-def layer_rms(inputs, out):
-    """RMS of every layer's own contribution y_l = x_{l+1} - x_l in the oracle's run."""
-    xs = list(inputs) + [out]
-    return [float(np.sqrt(np.mean((xs[l + 1] - xs[l]) ** 2))) for l in range(len(inputs))]
-
-
 def check_layers_one_by_one(lib, handles, which, inputs, out, n_launch):
     """Each GPU layer, fed the oracle's input of that layer, must reproduce the oracle's contribution
     of that layer within the layer tolerance.  The first rows of an n_launch-row batch carry the
@@ -117,14 +111,6 @@ def check_layers_one_by_one(lib, handles, which, inputs, out, n_launch):
         torch.cuda.synchronize()
         got = xd.cpu().numpy()[:rows].astype(np.float64) - xin[:rows].astype(np.float64)
         assert rel_err(got, xs[l + 1] - xs[l]) <= TOL_BF16, l
-
-
-def stack_tolerance(inputs, out):
-    """End-to-end bound for a deep stack, as a multiple of RMS(output): every layer's contribution
-    may be off by TOL_BF16 * RMS(y_l); the stack output is the sum of the contributions, so to first
-    order its error is bounded by the sum of those, and the later layers' response to the perturbed
-    stream (damped by RMSNorm, since the stream's RMS grows with depth) is allowed the same again."""
-    return 2.0 * TOL_BF16 * sum(layer_rms(inputs, out)) / float(np.sqrt(np.mean(out ** 2)))
 
 
 def destroy(lib, handles):
