@@ -350,13 +350,14 @@ int64_t tc_layer_schedule(int64_t n, int64_t d, int64_t Ipad, int bn, int ksplit
   const int n1 = static_cast<int>(Ipad / 128), n2 = static_cast<int>((d + bn - 1) / bn) * ksplit;   // down items per token block
   const int64_t cost_g = ((d + BK - 1) / BK) * kstep_cycles(256) + 1500;
   const int64_t cost_d = (Ipad / BK) * kstep_cycles(bn) / ksplit + 1500 + 24 * bn;     // + exposed part of the epilogue
-  // Group size.  At least enough token blocks to keep every pair busy on one pass over the weight
-  // tiles.  Weights that fit in L2 need no more (small groups finish their token blocks early, so
-  // down tiles become eligible early); larger weights are streamed from HBM once per group, so
-  // take at least 8 token blocks per pass.
+  // Group size.  Weights that fit in L2 can be re-read at will: take the token blocks one by one, so
+  // that they complete (and their down tiles become eligible) one by one.  Larger weights are
+  // streamed from HBM once per group: take enough token blocks to keep every pair busy on one pass
+  // over the weight tiles, and at least 8.
   int group = (pairs + n1 - 1) / n1 + 1;
   const bool weights_fit_l2 = 3 * d * Ipad * 2 <= (int64_t(48) << 20);
-  if (!weights_fit_l2 && group < 8) group = 8;
+  if (weights_fit_l2) group = 1;        // one token block after the other: blocks complete one by one, early
+  else if (group < 8) group = 8;
   if (group > m_pairs) group = m_pairs;
   std::vector<int32_t> g_order;
   g_order.reserve(static_cast<size_t>(m_pairs) * n1);
@@ -365,12 +366,31 @@ int64_t tc_layer_schedule(int64_t n, int64_t d, int64_t Ipad, int bn, int ksplit
       for (int m = g0; m < g0 + group && m < m_pairs; ++m) g_order.push_back(encode_tile(false, nb, m));
   std::vector<int64_t> avail(pairs, 0);
   std::vector<std::vector<int32_t>> lists(pairs);
+  if (weights_fit_l2) {
+    // Small layer: every gate|up tile (token block after token block), then every down item in the
+    // same block order, dealt round-robin.  Blocks complete progressively during the first phase, so
+    // by the time a pair reaches a down item its block has long been complete; the items are short
+    // enough (K slices) for the plain deal to balance.
+    int c = 0;
+    for (int32_t code : g_order) {
+      lists[c].push_back(code);
+      avail[c] += cost_g;
+      c = (c + 1) % pairs;
+    }
+    for (int m = 0; m < m_pairs; ++m)
+      for (int nb = 0; nb < n2; ++nb) {
+        lists[c].push_back(encode_tile(true, nb, m));
+        avail[c] += cost_d;
+        c = (c + 1) % pairs;
+      }
+    g_order.clear();
+  }
   std::vector<int> g_left(m_pairs, n1);
   std::vector<int64_t> block_done_at(m_pairs, 0);
   struct Ready { int64_t at; int32_t code; };
   std::vector<Ready> d_ready;          // FIFO of eligible down tiles
   size_t d_head = 0, g_next = 0;
-  const size_t total = static_cast<size_t>(m_pairs) * (n1 + n2);
+  const size_t total = weights_fit_l2 ? 0 : static_cast<size_t>(m_pairs) * (n1 + n2);
   size_t assigned = 0;
   // down tiles are the large items: no pair takes more than its share of them while gate|up tiles remain
   const int d_quota = static_cast<int>((static_cast<int64_t>(m_pairs) * n2 + pairs - 1) / pairs);
@@ -383,7 +403,9 @@ int64_t tc_layer_schedule(int64_t n, int64_t d, int64_t Ipad, int bn, int ksplit
         const int m = running[i].second;
         if (block_done_at[m] < running[i].first) block_done_at[m] = running[i].first;
         if (--g_left[m] == 0)
-          for (int nb = 0; nb < n2; ++nb) d_ready.push_back({block_done_at[m], encode_tile(true, nb, m)});
+          // eligible one gate|up tile time after the simulated completion: real tiles finish a little
+          // off the estimate, and a pair that reaches a down tile too early stalls on it
+          for (int nb = 0; nb < n2; ++nb) d_ready.push_back({block_done_at[m] + cost_g, encode_tile(true, nb, m)});
         running[i] = running.back();
         running.pop_back();
       } else {
@@ -398,7 +420,7 @@ int64_t tc_layer_schedule(int64_t n, int64_t d, int64_t Ipad, int bn, int ksplit
     int64_t now = avail[c];
     retire(now);
     int cd = -1;                         // the earliest-free pair that still has room for a down tile
-    if (d_head < d_ready.size()) {
+    if (d_head < d_ready.size() && (d_ready[d_head].at <= now || g_next >= g_order.size())) {
       for (int i = 0; i < pairs; ++i)
         if (d_taken[i] < d_quota && (cd < 0 || avail[i] < avail[cd])) cd = i;
       if (cd < 0 && g_next >= g_order.size()) cd = c;    // everyone has a share and nothing else is left
