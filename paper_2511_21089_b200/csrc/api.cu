@@ -294,9 +294,11 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
     a.y_bf16 = y_dtype == MLPMOE_BF16;
     a.n = n; a.d = h->d; a.Ipad = h->Ipad;
     const int m_blocks = static_cast<int>((h->d + 127) / 128);
-    int splits = h->num_sms / m_blocks;
-    if (splits > h->max_splits) splits = h->max_splits;
-    if (splits > h->Ipad / 64) splits = static_cast<int>(h->Ipad / 64);
+    a.accumulate = (residual == y && y_dtype == MLPMOE_FP32) ? 1 : 0;
+    // accumulate mode needs no staging buffer, so it can cut K finer (two work items per SM)
+    int splits = (a.accumulate ? 2 * h->num_sms : h->num_sms) / m_blocks;
+    if (!a.accumulate && splits > h->max_splits) splits = h->max_splits;
+    if (splits > h->Ipad / 64 / 8) splits = static_cast<int>(h->Ipad / 64 / 8);
     if (splits < 1) splits = 1;
     a.splits = splits;
     a.status = h->status;

@@ -13,6 +13,12 @@
 //
 // Warp roles as in the prefill kernels: warp 0 TMA producer, warp 1 TMEM owner + MMA issuer,
 // warps 2..5 epilogue.
+//
+// Back-to-back kernels: both kernels are launched with programmatic stream serialization, use
+// little enough shared memory (about 120 KB and 98 KB) and tensor memory (256 + 128 columns) for a
+// CTA of each to share an SM, and their producers start streaming WEIGHT tiles - which no earlier
+// kernel writes - before waiting for the previous kernel; only the activation tiles wait.  The
+// weight stream of the next kernel thus starts while the previous kernel drains.
 #include <cuda_bf16.h>
 
 #include "internal.h"
@@ -31,13 +37,13 @@ constexpr int MAXN = kDecodeMaxTokens;            // widest token tile
 // kernel 1: stage = 256 weight rows (128 gate + 128 up) + token tile
 constexpr int K1_W_BYTES = 256 * BK * 2;
 constexpr int K1_STAGE_BYTES = K1_W_BYTES + MAXN * BK * 2;
-constexpr int K1_STAGES = 5;
+constexpr int K1_STAGES = 3;
 constexpr int K1_BAR_OFFSET = K1_STAGES * K1_STAGE_BYTES;
 constexpr int K1_SMEM_BYTES = K1_BAR_OFFSET + 256 + 1024;
 // kernel 2: stage = 128 rows of WdT + activation tile
 constexpr int K2_W_BYTES = 128 * BK * 2;
 constexpr int K2_STAGE_BYTES = K2_W_BYTES + MAXN * BK * 2;
-constexpr int K2_STAGES = 8;
+constexpr int K2_STAGES = 4;
 constexpr int K2_BAR_OFFSET = K2_STAGES * K2_STAGE_BYTES;
 constexpr int K2_SMEM_BYTES = K2_BAR_OFFSET + 256 + 1024;
 
@@ -86,7 +92,6 @@ decode_gateup_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   griddep_launch_dependents();          // the next kernel may begin its set-up
-  griddep_wait();                       // inputs written by earlier kernels are complete and visible
   const uint32_t stage_tx = K1_W_BYTES + static_cast<uint32_t>(npad) * BK * 2;
 
   if (warp == 0) {
@@ -94,16 +99,34 @@ decode_gateup_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
       prefetch_tensormap(&tm_w);
       prefetch_tensormap(&tm_x);
       int stage = 0; uint32_t phase = 0; bool ok = true;
+      // weight tiles go out at once; the token tiles of those first stages follow once the kernel
+      // that writes X has completed
+      bool waited = false;
+      int deferred = 0, def_stage[K1_STAGES], def_kb[K1_STAGES];
+      auto flush = [&]() {
+        griddep_wait();
+        for (int i = 0; i < deferred; ++i)
+          tma_load_2d(smem + def_stage[i] * K1_STAGE_BYTES + K1_W_BYTES, &tm_x, def_kb[i] * BK, 0, &full_bar[def_stage[i]]);
+        waited = true;
+      };
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         for (int kb = 0; kb < num_k_blocks; ++kb) {
+          if (!waited && deferred == K1_STAGES) flush();
           if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* s = smem + stage * K1_STAGE_BYTES;
           mbar_expect_tx(&full_bar[stage], stage_tx);
           tma_load_2d(s, &tm_w, kb * BK, tile * 256, &full_bar[stage]);
-          tma_load_2d(s + K1_W_BYTES, &tm_x, kb * BK, 0, &full_bar[stage]);
+          if (waited) {
+            tma_load_2d(s + K1_W_BYTES, &tm_x, kb * BK, 0, &full_bar[stage]);
+          } else {
+            def_stage[deferred] = stage;
+            def_kb[deferred] = kb;
+            ++deferred;
+          }
           if (++stage == K1_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
+      if (!waited) flush();
     }
   } else if (warp == 1) {
     if (lane == 0) {
@@ -137,6 +160,7 @@ decode_gateup_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
       }
     }
   } else {
+    griddep_wait();                       // Hd may still be read by the previous layer's second kernel
     const int quad = warp % 4;
     int acc = 0; uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
@@ -175,7 +199,7 @@ decode_gateup_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 decode_down_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_constant__ CUtensorMap tm_h,
                    float* __restrict__ partial, uint32_t* __restrict__ counters, const float* R,
-                   void* Y, int y_bf16, int64_t n, int64_t d, int num_m_blocks, int splits,
+                   void* Y, int y_bf16, int accumulate, int64_t n, int64_t d, int num_m_blocks, int splits,
                    int total_k_blocks, int npad, uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align_1024(smem_raw);
@@ -200,7 +224,6 @@ decode_down_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   griddep_launch_dependents();          // the next kernel may begin its set-up
-  griddep_wait();                       // inputs written by earlier kernels are complete and visible
   const uint32_t stage_tx = K2_W_BYTES + static_cast<uint32_t>(npad) * BK * 2;
   const int num_items = num_m_blocks * splits;
 
@@ -210,19 +233,35 @@ decode_down_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_const
       prefetch_tensormap(&tm_wd);
       prefetch_tensormap(&tm_h);
       int stage = 0; uint32_t phase = 0; bool ok = true;
+      bool waited = false;                 // as in the first kernel: weights first, Hd tiles after the wait
+      int deferred = 0, def_stage[K2_STAGES], def_kb[K2_STAGES];
+      auto flush = [&]() {
+        griddep_wait();
+        for (int i = 0; i < deferred; ++i)
+          tma_load_2d(smem + def_stage[i] * K2_STAGE_BYTES + K2_W_BYTES, &tm_h, def_kb[i] * BK, 0, &full_bar[def_stage[i]]);
+        waited = true;
+      };
       for (int item = blockIdx.x; ok && item < num_items; item += gridDim.x) {
         const int m_blk = item % num_m_blocks, sp = item / num_m_blocks;
         const int kb0 = static_cast<int>(static_cast<int64_t>(sp) * total_k_blocks / splits);
         const int kb1 = static_cast<int>(static_cast<int64_t>(sp + 1) * total_k_blocks / splits);
         for (int kb = kb0; kb < kb1; ++kb) {
+          if (!waited && deferred == K2_STAGES) flush();
           if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* s = smem + stage * K2_STAGE_BYTES;
           mbar_expect_tx(&full_bar[stage], stage_tx);
           tma_load_2d(s, &tm_wd, kb * BK, m_blk * 128, &full_bar[stage]);
-          tma_load_2d(s + K2_W_BYTES, &tm_h, kb * BK, 0, &full_bar[stage]);
+          if (waited) {
+            tma_load_2d(s + K2_W_BYTES, &tm_h, kb * BK, 0, &full_bar[stage]);
+          } else {
+            def_stage[deferred] = stage;
+            def_kb[deferred] = kb;
+            ++deferred;
+          }
           if (++stage == K2_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
+      if (!waited) flush();
     }
   } else if (warp == 1) {
     if (lane == 0) {
@@ -255,6 +294,7 @@ decode_down_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_const
       }
     }
   } else {
+    griddep_wait();                       // partial sums, counters and Y belong to earlier kernels until now
     const int quad = warp % 4;
     int acc = 0; uint32_t acc_phase = 0;
     for (int item = blockIdx.x; item < num_items; item += gridDim.x) {
@@ -280,6 +320,15 @@ decode_down_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_const
       }
       const int64_t m = static_cast<int64_t>(m_blk) * 128 + quad * 32 + lane;    // output feature of this thread
       const bool m_ok = m < d;
+      if (accumulate) {
+        // Y (fp32) already holds the residual: every slice adds its part, no staging and no hand-over
+        if (m_ok) {
+#pragma unroll
+          for (int t = 0; t < MAXN; ++t)
+            if (t < n) atomicAdd(static_cast<float*>(Y) + static_cast<int64_t>(t) * d + m, v[t]);
+        }
+        continue;
+      }
       // 1. publish this slice's partial row
       if (m_ok) {
         float4* dst = reinterpret_cast<float4*>(partial + (static_cast<int64_t>(sp) * d + m) * npad);
@@ -359,7 +408,7 @@ cudaError_t launch_decode_down(const DecodeArgs& a, int num_sms, cudaStream_t st
   const int items = m_blocks * a.splits;
   const int grid2 = items < num_sms ? items : num_sms;
   return launch_pdl(decode_down_kernel, dim3(grid2), dim3(NUM_THREADS), K2_SMEM_BYTES, st, a.tm_wd, a.tm_h, a.partial, a.counters,
-                    a.R, a.Y, a.y_bf16, a.n, a.d, m_blocks, a.splits, static_cast<int>(a.Ipad / BK), a.npad, a.status);
+                    a.R, a.Y, a.y_bf16, a.accumulate, a.n, a.d, m_blocks, a.splits, static_cast<int>(a.Ipad / BK), a.npad, a.status);
 }
 
 }  // namespace mlpmoe

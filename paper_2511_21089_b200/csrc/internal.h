@@ -141,6 +141,7 @@ struct DecodeArgs {
   int y_bf16;
   int64_t n, d, Ipad;
   int npad, splits;
+  int accumulate;       // 1: Y (fp32) already holds the residual and every K slice adds into it
   uint32_t* status;
 };
 cudaError_t launch_decode_gateup(const DecodeArgs& a, int num_sms, cudaStream_t st);
