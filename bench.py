@@ -87,12 +87,12 @@ def layer_inputs(layer: int, w):
     return bits, d_b, alpha, keep
 
 
-# DRAM traffic of one gate|up launch from the ncu capture summarised in
-# profiles/tc_pair_gemm_qwen_c2_2layers.md (dram__bytes_read.sum + dram__bytes_write.sum), valid
+# DRAM traffic of one fused layer-kernel launch from the ncu capture summarised in
+# profiles/tc_layer_kernel_qwen_c2_2layers.md (dram__bytes_read.sum + dram__bytes_write.sum), valid
 # only while the kernel's sources are the ones that were profiled.
-GATEUP_TRAFFIC_BYTES = 20.70e6 + 0.12e6
+GATEUP_TRAFFIC_BYTES = 42.16e6 + 4.08e6
 GATEUP_SOURCES = ("tc_layer.cu", "tc_common.cuh", "ptx.cuh")
-GATEUP_SOURCES_SHA = "b842eb5204afc5ef"
+GATEUP_SOURCES_SHA = "058b6e7cb57620d0"
 
 
 def gateup_traffic():
