@@ -170,6 +170,29 @@ def run_reference(args):
     print(json.dumps(out))
 
 
+# ------------------------------------------------------------- multi-rank glue --
+def rank_batch(cfg: int, n: int, d: int, rank: int) -> np.ndarray:
+    """Token split: every rank draws its own n-token batch (rows are independent, so the path
+    shards by tokens with no collective on the data path)."""
+    return synth.tokens(cfg, n, d, stream=rank)
+
+
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a few per-rank timings over all ranks (the job is as slow as its
+    slowest rank); a no-op outside torch.distributed."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def job_throughput(world: int, n: int, steps: int, ms_total_max: float) -> float:
+    """Whole-job tokens/s: all ranks' tokens over the slowest rank's time."""
+    return world * n * steps / (ms_total_max * 1e-3)
+
+
 # ------------------------------------------------------------------- CUDA leg --
 class ClockSampler:
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -253,7 +276,7 @@ def run_ours(args):
         del dev
     torch.cuda.synchronize()
 
-    x_f32 = synth.tokens(w["cfg"], n, d, stream=rank)                                 # each rank its own batch
+    x_f32 = rank_batch(w["cfg"], n, d, rank)
     y_host = torch.empty((n, d), dtype=torch.float32).pin_memory()
     if w["stack"]:
         x0_host = torch.from_numpy(x_f32).pin_memory()
@@ -335,12 +358,9 @@ def run_ours(args):
     if not np.isfinite(y_host.numpy()).all():
         raise RuntimeError("non-finite output")
 
-    t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = float(t[0]), float(t[1])
+    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms], device="cuda")
     ms_step = ms_total / args.steps
-    value = world * n * args.steps / (ms_total * 1e-3)
+    value = job_throughput(world, n, args.steps, ms_total)
 
     if rank == 0:
         pk = peaks()
