@@ -172,7 +172,6 @@ struct mlpmoe_layer_s {
   void* fade_work = nullptr;
   float* partial = nullptr;
   uint32_t* counters = nullptr;
-  float* rowstat = nullptr;                                 // [2 x 64] squared row norms of the chained decode stack
   uint32_t* block_done = nullptr;                           // [2 x ceil(max_tokens / 256)] gate|up completion counters
   int64_t max_blocks = 0;
   int32_t* tile_sched = nullptr;                            // device: tile sequences + offsets of the fused prefill kernel
@@ -213,7 +212,7 @@ void free_layer(mlpmoe_layer_s* h) {
   cudaFree(h->Wg_c); cudaFree(h->Wu_c); cudaFree(h->Wd_c);
   cudaFree(h->Wgu); cudaFree(h->WdT);
   cudaFree(h->scale); cudaFree(h->src_row); cudaFree(h->row_nnz);
-  cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->block_done); cudaFree(h->tile_sched); cudaFree(h->rowstat); cudaFree(h->status);
+  cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->block_done); cudaFree(h->tile_sched); cudaFree(h->status);
   ws_release(h->ws);
   delete h;
 }
@@ -259,17 +258,8 @@ mlpmoe_status_t reschedule(mlpmoe_layer_s* h, cudaStream_t st) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Optional link of a chained decode stack: the layer reads the un-normalised bf16 stream plus its
-// squared row norms and leaves the same pair behind for the next layer.
-struct DecodeChain {
-  const float* sumsq_in;
-  float* sumsq_next;
-  void* xb_next;
-  float eps;
-};
-
 mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t n, const float* residual,
-                             mlpmoe_dtype_t y_dtype, cudaStream_t st, const DecodeChain* chain = nullptr) {
+                             mlpmoe_dtype_t y_dtype, cudaStream_t st) {
   if (!h || n < 0) return MLPMOE_ERR_INVALID_ARG;
   if (n == 0) return MLPMOE_OK;
   if (!x || !y || n > h->max_tokens || !aligned16(x) || !aligned16(y) || (residual && !aligned16(residual)))
@@ -305,10 +295,6 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
     a.n = n; a.d = h->d; a.Ipad = h->Ipad;
     const int m_blocks = static_cast<int>((h->d + 127) / 128);
     a.accumulate = (residual == y && y_dtype == MLPMOE_FP32) ? 1 : 0;
-    a.sumsq_in = chain ? chain->sumsq_in : nullptr;
-    a.sumsq_next = chain ? chain->sumsq_next : nullptr;
-    a.xb_next = chain ? chain->xb_next : nullptr;
-    a.eps = chain ? chain->eps : 0.f;
     // accumulate mode needs no staging buffer, so it can cut K finer (two work items per SM)
     int splits = (a.accumulate ? 2 * h->num_sms : h->num_sms) / m_blocks;
     if (!a.accumulate && splits > h->max_splits) splits = h->max_splits;
@@ -482,7 +468,6 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
        cudaMalloc(&h->fade_work, fade_work_bytes(2 * B)) == cudaSuccess &&
        cudaMalloc(&h->partial, sizeof(float) * static_cast<size_t>(h->max_splits) * d_model * kDecodeMaxTokens) == cudaSuccess &&
        cudaMalloc(&h->counters, sizeof(uint32_t) * m_blocks * 4) == cudaSuccess &&
-       cudaMalloc(reinterpret_cast<void**>(&h->rowstat), sizeof(float) * 2 * kDecodeMaxTokens) == cudaSuccess &&
        cudaMalloc(&h->block_done, sizeof(uint32_t) * 2 * h->max_blocks) == cudaSuccess &&
        cudaMalloc(&h->tile_sched, sizeof(int32_t) * h->sched_capacity) == cudaSuccess &&
        cudaMalloc(&h->status, sizeof(uint32_t)) == cudaSuccess &&
@@ -617,31 +602,6 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
   if (n == 0) return MLPMOE_OK;
   if (!x || !aligned16(x)) return MLPMOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (layers[0]->dtype == MLPMOE_BF16 && n <= kDecodeMaxTokens) {
-    // Decode: no RMSNorm kernel between the layers.  The normalisation factor of a token row is a
-    // scalar, so it is applied to the pre-activations in the first kernel's epilogue, and the second
-    // kernel of each layer leaves the bf16 copy of the updated stream and its squared row norms for
-    // the next layer.
-    mlpmoe_layer_s* h0 = layers[0];
-    pdl_overlap_enabled() = !h0->timing;
-    const long e0 = rec_event(h0, st);
-    CK(launch_decode_prep(x, h0->ws->xnorm, h0->rowstat, n, h0->d, st));
-    const long e1 = rec_event(h0, st);
-    add_span(h0, SPAN_RMSNORM, e0, e1);
-    h0->launches += 1;
-    const void* xb = h0->ws->xnorm;
-    for (int l = 0; l < n_layers; ++l) {
-      mlpmoe_layer_s* h = layers[l];
-      DecodeChain c;
-      c.sumsq_in = h0->rowstat + (l % 2) * kDecodeMaxTokens;
-      c.sumsq_next = h0->rowstat + ((l + 1) % 2) * kDecodeMaxTokens;
-      c.xb_next = h0->ws->xnorm;
-      c.eps = eps;
-      rc = forward_impl(h, xb, x, n, x, MLPMOE_FP32, st, &c);
-      if (rc != MLPMOE_OK) return rc;
-    }
-    return MLPMOE_OK;
-  }
   for (int l = 0; l < n_layers; ++l) {
     mlpmoe_layer_s* h = layers[l];
     pdl_overlap_enabled() = !h->timing;

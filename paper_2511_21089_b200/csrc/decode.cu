@@ -68,8 +68,7 @@ __device__ __forceinline__ void load_acc_row(uint32_t taddr, int npad, float (&v
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 decode_gateup_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
                      const float* __restrict__ scale, __nv_bfloat16* __restrict__ Hd, int64_t n, int64_t Ipad,
-                     int num_tiles, int num_k_blocks, int npad, const float* __restrict__ sumsq_in,
-                     float* __restrict__ sumsq_clear, float inv_d, float eps, uint32_t* status) {
+                     int num_tiles, int num_k_blocks, int npad, uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align_1024(smem_raw);
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + K1_BAR_OFFSET);
@@ -164,12 +163,6 @@ decode_gateup_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
     griddep_wait();                       // Hd may still be read by the previous layer's second kernel
     const int quad = warp % 4;
     int acc = 0; uint32_t acc_phase = 0;
-    // chained stack mode: X holds the un-normalised stream and sumsq_in the squared row norms, so the
-    // RMSNorm factor of token t is applied to both pre-activations here (it commutes with the GEMM);
-    // sumsq_clear is the buffer the second kernel of this layer will accumulate the next norms into
-    if (sumsq_clear != nullptr && blockIdx.x == 0 && warp == 2) {
-      for (int t = lane; t < n; t += 32) sumsq_clear[t] = 0.f;
-    }
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
       bool ok = mbar_wait_bounded(&tfull_bar[acc], acc_phase, abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);
@@ -187,9 +180,8 @@ decode_gateup_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
 #pragma unroll
       for (int t = 0; t < MAXN; ++t) {
         if (t < n) {
-          const float r = sumsq_in != nullptr ? rsqrtf(__ldg(sumsq_in + t) * inv_d + eps) : 1.0f;
-          const float gv = g[t] * r;
-          const float h = __fdividef(gv, 1.0f + __expf(-gv)) * (u[t] * r) * sc;
+          const float gv = g[t];
+          const float h = __fdividef(gv, 1.0f + __expf(-gv)) * u[t] * sc;
           Hd[static_cast<int64_t>(t) * Ipad + j] = __float2bfloat16_rn(h);
         }
       }
@@ -208,8 +200,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 decode_down_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_constant__ CUtensorMap tm_h,
                    float* __restrict__ partial, uint32_t* __restrict__ counters, const float* R,
                    void* Y, int y_bf16, int accumulate, int64_t n, int64_t d, int num_m_blocks, int splits,
-                   int total_k_blocks, int npad, __nv_bfloat16* __restrict__ xb_next, float* __restrict__ sumsq_next,
-                   uint32_t* status) {
+                   int total_k_blocks, int npad, uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align_1024(smem_raw);
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + K2_BAR_OFFSET);
@@ -336,34 +327,6 @@ decode_down_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_const
           for (int t = 0; t < MAXN; ++t)
             if (t < n) atomicAdd(static_cast<float*>(Y) + static_cast<int64_t>(t) * d + m, v[t]);
         }
-        if (xb_next != nullptr) {
-          // chained stack mode: the warp that adds the last slice of these 32 output features reads
-          // the finished values back and prepares the next layer's input: bf16 copy of the stream and
-          // this group's share of every token's squared norm
-          __threadfence();
-          __syncwarp();
-          uint32_t seen = 0;
-          if (lane == 0) seen = atomicAdd(&counters[m_blk * 4 + quad], 1u);
-          seen = __shfl_sync(0xFFFFFFFFu, seen, 0);
-          if (seen == static_cast<uint32_t>(splits - 1)) {
-            __threadfence();
-            float xv[MAXN];
-#pragma unroll
-            for (int t = 0; t < MAXN; ++t)
-              xv[t] = (t < n && m_ok) ? __ldcg(static_cast<const float*>(Y) + static_cast<int64_t>(t) * d + m) : 0.f;
-#pragma unroll
-            for (int t = 0; t < MAXN; ++t) {
-              if (t < n) {
-                if (m_ok) xb_next[static_cast<int64_t>(t) * d + m] = __float2bfloat16_rn(xv[t]);
-                float sq = xv[t] * xv[t];
-                for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, o);
-                if (lane == 0) atomicAdd(sumsq_next + t, sq);
-              }
-            }
-            __syncwarp();
-            if (lane == 0) counters[m_blk * 4 + quad] = 0;    // ready for the next call
-          }
-        }
         continue;
       }
       // 1. publish this slice's partial row
@@ -422,36 +385,7 @@ decode_down_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_const
   if (threadIdx.x == 0 && *abort_flag) atomicExch(status, kStatusTimeout);
 }
 
-// Start of a chained decode stack: bf16 copy of the fp32 stream (un-normalised) and the squared
-// norm of every token row.  One block per row.
-__global__ void __launch_bounds__(256) decode_prep_kernel(const float* __restrict__ x, __nv_bfloat16* __restrict__ xb,
-                                                          float* __restrict__ sumsq, int64_t d) {
-  const int64_t t = blockIdx.x;
-  griddep_launch_dependents();
-  griddep_wait();
-  float ss = 0.f;
-  for (int64_t k = threadIdx.x; k < d; k += blockDim.x) {
-    const float v = x[t * d + k];
-    xb[t * d + k] = __float2bfloat16_rn(v);
-    ss += v * v;
-  }
-  __shared__ float red[8];
-  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
-  if (threadIdx.x % 32 == 0) red[threadIdx.x / 32] = ss;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    float tot = 0.f;
-    for (int i = 0; i < 8; ++i) tot += red[i];
-    sumsq[t] = tot;
-  }
-}
-
 }  // namespace
-
-cudaError_t launch_decode_prep(const float* x, void* xb, float* sumsq, int64_t n, int64_t d, cudaStream_t st) {
-  if (n == 0) return cudaSuccess;
-  return launch_pdl(decode_prep_kernel, dim3(static_cast<unsigned>(n)), dim3(256), 0, st, x, static_cast<__nv_bfloat16*>(xb), sumsq, d);
-}
 
 cudaError_t decode_init() {
   cudaError_t e = cudaFuncSetAttribute(decode_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, K1_SMEM_BYTES);
@@ -465,8 +399,7 @@ cudaError_t launch_decode_gateup(const DecodeArgs& a, int num_sms, cudaStream_t 
   const int kb1 = static_cast<int>((a.d + BK - 1) / BK);
   const int grid1 = tiles1 < num_sms ? tiles1 : num_sms;
   return launch_pdl(decode_gateup_kernel, dim3(grid1), dim3(NUM_THREADS), K1_SMEM_BYTES, st, a.tm_w, a.tm_x, a.scale,
-                    static_cast<__nv_bfloat16*>(a.Hd), a.n, a.Ipad, tiles1, kb1, a.npad, a.sumsq_in, a.sumsq_next,
-                    1.0f / static_cast<float>(a.d), a.eps, a.status);
+                    static_cast<__nv_bfloat16*>(a.Hd), a.n, a.Ipad, tiles1, kb1, a.npad, a.status);
 }
 
 cudaError_t launch_decode_down(const DecodeArgs& a, int num_sms, cudaStream_t st) {
@@ -475,8 +408,7 @@ cudaError_t launch_decode_down(const DecodeArgs& a, int num_sms, cudaStream_t st
   const int items = m_blocks * a.splits;
   const int grid2 = items < num_sms ? items : num_sms;
   return launch_pdl(decode_down_kernel, dim3(grid2), dim3(NUM_THREADS), K2_SMEM_BYTES, st, a.tm_wd, a.tm_h, a.partial, a.counters,
-                    a.R, a.Y, a.y_bf16, a.accumulate, a.n, a.d, m_blocks, a.splits, static_cast<int>(a.Ipad / BK), a.npad,
-                    static_cast<__nv_bfloat16*>(a.xb_next), a.sumsq_next, a.status);
+                    a.R, a.Y, a.y_bf16, a.accumulate, a.n, a.d, m_blocks, a.splits, static_cast<int>(a.Ipad / BK), a.npad, a.status);
 }
 
 }  // namespace mlpmoe

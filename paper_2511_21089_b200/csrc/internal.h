@@ -142,17 +142,10 @@ struct DecodeArgs {
   int64_t n, d, Ipad;
   int npad, splits;
   int accumulate;       // 1: Y (fp32) already holds the residual and every K slice adds into it
-  // chained stack mode (all null otherwise): X is the un-normalised bf16 stream, sumsq_in its squared
-  // row norms; the second kernel leaves the next layer's bf16 stream and squared norms behind
-  const float* sumsq_in;
-  float* sumsq_next;
-  void* xb_next;
-  float eps;
   uint32_t* status;
 };
 cudaError_t launch_decode_gateup(const DecodeArgs& a, int num_sms, cudaStream_t st);
 cudaError_t launch_decode_down(const DecodeArgs& a, int num_sms, cudaStream_t st);
-cudaError_t launch_decode_prep(const float* x, void* xb, float* sumsq, int64_t n, int64_t d, cudaStream_t st);
 cudaError_t decode_init();
 
 }  // namespace mlpmoe
