@@ -33,7 +33,6 @@ constexpr int BK = 64;
 constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
 constexpr int MAXN = kDecodeMaxTokens;            // widest token tile
-constexpr int L2_AHEAD = 8;                       // weight K-steps requested into L2 ahead of the shared-memory ring
 
 // kernel 1: stage = 256 weight rows (128 gate + 128 up) + token tile
 constexpr int K1_W_BYTES = 256 * BK * 2;
@@ -111,12 +110,7 @@ decode_gateup_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
         waited = true;
       };
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-        // The ring holds only a few K-steps (two kernels share the SM's shared memory), so HBM would
-        // idle whenever this CTA is blocked on the previous kernel: keep L2_AHEAD further weight
-        // K-steps on their way into L2.
-        for (int kb = 0; kb < L2_AHEAD && kb < num_k_blocks; ++kb) tma_prefetch_l2_2d(&tm_w, kb * BK, tile * 256);
         for (int kb = 0; kb < num_k_blocks; ++kb) {
-          if (kb + L2_AHEAD < num_k_blocks) tma_prefetch_l2_2d(&tm_w, (kb + L2_AHEAD) * BK, tile * 256);
           if (!waited && deferred == K1_STAGES) flush();
           if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* s = smem + stage * K1_STAGE_BYTES;
@@ -251,9 +245,7 @@ decode_down_kernel(const __grid_constant__ CUtensorMap tm_wd, const __grid_const
         const int m_blk = item % num_m_blocks, sp = item / num_m_blocks;
         const int kb0 = static_cast<int>(static_cast<int64_t>(sp) * total_k_blocks / splits);
         const int kb1 = static_cast<int>(static_cast<int64_t>(sp + 1) * total_k_blocks / splits);
-        for (int kb = kb0; kb < kb0 + L2_AHEAD && kb < kb1; ++kb) tma_prefetch_l2_2d(&tm_wd, kb * BK, m_blk * 128);
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (kb + L2_AHEAD < kb1) tma_prefetch_l2_2d(&tm_wd, (kb + L2_AHEAD) * BK, m_blk * 128);
           if (!waited && deferred == K2_STAGES) flush();
           if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* s = smem + stage * K2_STAGE_BYTES;
