@@ -171,6 +171,9 @@ struct mlpmoe_layer_s {
   Workspace* ws = nullptr;
   void* fade_work = nullptr;
   float* partial = nullptr;
+  DecodeStackLayer* stack_dev = nullptr;                    // layer records of the persistent decode-stack kernel
+  uint32_t* stack_counter = nullptr;                        // its grid-wide event counter
+  std::vector<DecodeStackLayer> stack_host;                 // what stack_dev currently holds
   uint32_t* counters = nullptr;
   uint32_t* block_done = nullptr;                           // [2 x ceil(max_tokens / 256)] gate|up completion counters
   int64_t max_blocks = 0;
@@ -194,6 +197,7 @@ struct mlpmoe_layer_s {
 namespace {
 
 constexpr size_t kEventPool = 2048;
+constexpr int kMaxStackLayers = 256;       // layers one persistent decode-stack launch can take
 enum { SPAN_GATEUP = 0, SPAN_DOWN = 1, SPAN_RMSNORM = 2 };
 
 // Records an event on `st` and returns its index in the pool, or -1 when timing is off / the pool is used up.
@@ -212,7 +216,7 @@ void free_layer(mlpmoe_layer_s* h) {
   cudaFree(h->Wg_c); cudaFree(h->Wu_c); cudaFree(h->Wd_c);
   cudaFree(h->Wgu); cudaFree(h->WdT);
   cudaFree(h->scale); cudaFree(h->src_row); cudaFree(h->row_nnz);
-  cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->block_done); cudaFree(h->tile_sched); cudaFree(h->status);
+  cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->block_done); cudaFree(h->tile_sched); cudaFree(h->stack_dev); cudaFree(h->stack_counter); cudaFree(h->status);
   ws_release(h->ws);
   delete h;
 }
@@ -387,6 +391,16 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
   return MLPMOE_OK;
 }
 
+// The persistent decode-stack kernel needs one CTA of it to fit on every SM (checked once).
+bool stack_kernel_ok() {
+  static int state = -1;
+  if (state < 0) {
+    int per_sm = 0;
+    state = (decode_stack_init(&per_sm) == cudaSuccess && per_sm >= 1) ? 1 : 0;
+  }
+  return state == 1;
+}
+
 mlpmoe_status_t check_stack(const mlpmoe_handle_t* layers, int32_t n_layers, int64_t n) {
   if (!layers || n_layers <= 0 || n < 0) return MLPMOE_ERR_INVALID_ARG;
   for (int l = 0; l < n_layers; ++l) {
@@ -468,6 +482,8 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
        cudaMalloc(&h->fade_work, fade_work_bytes(2 * B)) == cudaSuccess &&
        cudaMalloc(&h->partial, sizeof(float) * static_cast<size_t>(h->max_splits) * d_model * kDecodeMaxTokens) == cudaSuccess &&
        cudaMalloc(&h->counters, sizeof(uint32_t) * m_blocks * 4) == cudaSuccess &&
+       cudaMalloc(reinterpret_cast<void**>(&h->stack_dev), sizeof(DecodeStackLayer) * kMaxStackLayers) == cudaSuccess &&
+       cudaMalloc(reinterpret_cast<void**>(&h->stack_counter), sizeof(uint32_t)) == cudaSuccess &&
        cudaMalloc(&h->block_done, sizeof(uint32_t) * 2 * h->max_blocks) == cudaSuccess &&
        cudaMalloc(&h->tile_sched, sizeof(int32_t) * h->sched_capacity) == cudaSuccess &&
        cudaMalloc(&h->status, sizeof(uint32_t)) == cudaSuccess &&
@@ -602,6 +618,38 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
   if (n == 0) return MLPMOE_OK;
   if (!x || !aligned16(x)) return MLPMOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (layers[0]->dtype == MLPMOE_BF16 && n <= kDecodeMaxTokens && n_layers <= kMaxStackLayers && layers[0]->d <= 32768 &&
+      stack_kernel_ok()) {
+    // decode: the whole stack in one persistent kernel (weights keep streaming across layer boundaries)
+    mlpmoe_layer_s* h0 = layers[0];
+    const int npad = n <= 16 ? 16 : (n <= 32 ? 32 : 64);
+    std::vector<DecodeStackLayer> recs(static_cast<size_t>(n_layers));
+    std::memset(recs.data(), 0, sizeof(DecodeStackLayer) * recs.size());
+    for (int l = 0; l < n_layers; ++l) {
+      mlpmoe_layer_s* h = layers[l];
+      recs[l].tm_wgu = h->tm_wgu;
+      recs[l].tm_wdt = h->tm_wdt;
+      if (!make_tmap(&recs[l].tm_hd, h->ws->H, h->Ipad, n, h->Ipad, npad)) return MLPMOE_ERR_CUDA;
+      recs[l].scale = h->scale;
+      recs[l].Hd = static_cast<__nv_bfloat16*>(h->ws->H);
+      recs[l].Ipad = static_cast<int32_t>(h->Ipad);
+    }
+    if (h0->stack_host.size() != recs.size() ||
+        std::memcmp(h0->stack_host.data(), recs.data(), sizeof(DecodeStackLayer) * recs.size()) != 0) {
+      h0->stack_host = recs;
+      CK(cudaMemcpyAsync(h0->stack_dev, h0->stack_host.data(), sizeof(DecodeStackLayer) * recs.size(), cudaMemcpyHostToDevice, st));
+    }
+    CUtensorMap tm_x;
+    if (!make_tmap(&tm_x, h0->ws->xnorm, h0->d, n, h0->d, npad)) return MLPMOE_ERR_CUDA;
+    CK(cudaMemsetAsync(h0->stack_counter, 0, sizeof(uint32_t), st));
+    const long e0 = rec_event(h0, st);
+    CK(launch_decode_stack(h0->stack_dev, n_layers, tm_x, x, h0->ws->xnorm, n, h0->d, npad, eps, h0->stack_counter, h0->status,
+                           h0->num_sms, st));
+    const long e1 = rec_event(h0, st);
+    add_span(h0, SPAN_GATEUP, e0, e1);
+    h0->launches += 1;
+    return MLPMOE_OK;
+  }
   for (int l = 0; l < n_layers; ++l) {
     mlpmoe_layer_s* h = layers[l];
     pdl_overlap_enabled() = !h->timing;

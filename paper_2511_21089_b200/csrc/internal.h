@@ -1,6 +1,7 @@
 // Internal launch interface between the C-ABI host code and the kernel files.
 #pragma once
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -147,5 +148,21 @@ struct DecodeArgs {
 cudaError_t launch_decode_gateup(const DecodeArgs& a, int num_sms, cudaStream_t st);
 cudaError_t launch_decode_down(const DecodeArgs& a, int num_sms, cudaStream_t st);
 cudaError_t decode_init();
+
+// ----------------------------------------------------------- decode_stack.cu --
+// One record per layer of a decode stack, read by the persistent stack kernel from device memory.
+struct alignas(64) DecodeStackLayer {
+  CUtensorMap tm_wgu;    // Wgu [2 Ipad x d]  box 64 x 256
+  CUtensorMap tm_wdt;    // WdT [d x Ipad]    box 64 x 128
+  CUtensorMap tm_hd;     // Hd  [n x Ipad]    box 64 x npad
+  const float* scale;    // [Ipad]
+  __nv_bfloat16* Hd;     // [n x Ipad]
+  int32_t Ipad;
+  int32_t pad_[11];
+};
+cudaError_t decode_stack_init(int* max_ctas_per_sm);
+cudaError_t launch_decode_stack(const DecodeStackLayer* layers_dev, int n_layers, const CUtensorMap& tm_x, float* x, void* xnorm,
+                                int64_t n, int64_t d, int npad, float eps, uint32_t* event_counter, uint32_t* status,
+                                int num_sms, cudaStream_t st);
 
 }  // namespace mlpmoe
