@@ -483,7 +483,7 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
        cudaMalloc(&h->partial, sizeof(float) * static_cast<size_t>(h->max_splits) * d_model * kDecodeMaxTokens) == cudaSuccess &&
        cudaMalloc(&h->counters, sizeof(uint32_t) * m_blocks * 4) == cudaSuccess &&
        cudaMalloc(reinterpret_cast<void**>(&h->stack_dev), sizeof(DecodeStackLayer) * kMaxStackLayers) == cudaSuccess &&
-       cudaMalloc(reinterpret_cast<void**>(&h->stack_counter), sizeof(uint32_t)) == cudaSuccess &&
+       cudaMalloc(reinterpret_cast<void**>(&h->stack_counter), sizeof(uint32_t) * 3 * kMaxStackLayers) == cudaSuccess &&
        cudaMalloc(&h->block_done, sizeof(uint32_t) * 2 * h->max_blocks) == cudaSuccess &&
        cudaMalloc(&h->tile_sched, sizeof(int32_t) * h->sched_capacity) == cudaSuccess &&
        cudaMalloc(&h->status, sizeof(uint32_t)) == cudaSuccess &&
@@ -641,7 +641,7 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
     }
     CUtensorMap tm_x;
     if (!make_tmap(&tm_x, h0->ws->xnorm, h0->d, n, h0->d, npad)) return MLPMOE_ERR_CUDA;
-    CK(cudaMemsetAsync(h0->stack_counter, 0, sizeof(uint32_t), st));
+    CK(cudaMemsetAsync(h0->stack_counter, 0, sizeof(uint32_t) * 3 * n_layers, st));
     const long e0 = rec_event(h0, st);
     CK(launch_decode_stack(h0->stack_dev, n_layers, tm_x, x, h0->ws->xnorm, n, h0->d, npad, eps, h0->stack_counter, h0->status,
                            h0->num_sms, st));

@@ -41,8 +41,10 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
 }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// Events are numbered in program order: 3 per layer (N, A, B).  Event e has happened once the
-// counter has reached (e + 1) * arrivals_per_event.
+// Events are numbered in program order, 3 per layer (N, A, B), and each has its own arrival counter
+// (a CTA without work in a phase arrives at once, so one shared counter would let early arrivals
+// at later events stand in for missing arrivals at earlier ones).  Event e has happened once
+// counter[e] has reached arrivals_per_event.
 __device__ __forceinline__ bool event_passed(const uint32_t* counter, uint32_t target) {
   return ld_acquire_u32(counter) >= target;
 }
@@ -137,7 +139,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
       // activation tiles that wait for the current gating event: (stage, tensor map, K-step)
       int deferred = 0, def_stage[STAGES], def_kb[STAGES];
       const CUtensorMap* def_map = nullptr;
-      uint32_t gate_target = 0;            // counter value at which the gating event has happened
+      const uint32_t* gate = event_counter;  // counter of the gating event
       bool gate_open = false;
       auto flush = [&]() {
         fence_async_proxy();               // what the acquire made visible must be seen by the TMA reads
@@ -148,8 +150,8 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
       };
       // issues one stage: weights at once, the token tile as soon as the gate is open
       auto issue = [&](const CUtensorMap* wmap, int wrow, uint32_t wbytes, const CUtensorMap* amap, int kb) -> bool {
-        if (!gate_open && (deferred == STAGES || event_passed(event_counter, gate_target))) {
-          if (deferred == STAGES && !event_wait(event_counter, gate_target, abort_flag)) return false;
+        if (!gate_open && (deferred == STAGES || event_passed(gate, per_event))) {
+          if (deferred == STAGES && !event_wait(gate, per_event, abort_flag)) return false;
           flush();
         }
         if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, WAIT_NS)) return false;
@@ -168,22 +170,22 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
         const DecodeStackLayer* L = layers + l;
         const int Ipad = L->Ipad;
         // phase A needs event N(l): index 3l
-        if (deferred > 0) { if (!event_wait(event_counter, gate_target, abort_flag)) { ok = false; break; } flush(); }
-        gate_target = static_cast<uint32_t>(3 * l + 1) * per_event; gate_open = false; def_map = &tm_x;
+        if (deferred > 0) { if (!event_wait(gate, per_event, abort_flag)) { ok = false; break; } flush(); }
+        gate = event_counter + 3 * l; gate_open = false; def_map = &tm_x;
         for (int tile = cta; ok && tile < Ipad / 128; tile += ctas)
           for (int kb = 0; kb < kb1; ++kb)
             if (!issue(&L->tm_wgu, tile * 256, W_BYTES, &tm_x, kb)) { ok = false; break; }
         if (!ok) break;
         // phase B needs event A(l): index 3l + 1
-        if (deferred > 0) { if (!event_wait(event_counter, gate_target, abort_flag)) { ok = false; break; } flush(); }
-        gate_target = static_cast<uint32_t>(3 * l + 2) * per_event; gate_open = false; def_map = &L->tm_hd;
+        if (deferred > 0) { if (!event_wait(gate, per_event, abort_flag)) { ok = false; break; } flush(); }
+        gate = event_counter + 3 * l + 1; gate_open = false; def_map = &L->tm_hd;
         BItem it[4];
         const int nit = b_items(cta, ctas, m_blocks, Ipad / BK, it);
         for (int i = 0; ok && i < nit; ++i)
           for (int kb = it[i].kb_lo; kb < it[i].kb_hi; ++kb)
             if (!issue(&L->tm_wdt, it[i].m_blk * 128, W_BYTES / 2, &L->tm_hd, kb)) { ok = false; break; }
       }
-      if (ok && deferred > 0 && event_wait(event_counter, gate_target, abort_flag)) flush();
+      if (ok && deferred > 0 && event_wait(gate, per_event, abort_flag)) flush();
     }
   }
   else if (warp == 1) {
@@ -231,10 +233,10 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
     const int quad = warp % 4;
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
-    auto arrive_event = [&]() {            // this warp's part of the phase is written and visible
+    auto arrive_event = [&](int e) {       // this warp's part of the phase is written and visible
       __threadfence();
       __syncwarp();
-      if (lane == 0) atomicAdd(event_counter, 1u);
+      if (lane == 0) atomicAdd(event_counter + e, 1u);
     };
     auto wait_acc = [&]() -> bool {
       bool w = mbar_wait_bounded(&tfull_bar[acc], acc_phase, abort_flag, WAIT_NS);
@@ -254,7 +256,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
       const int Ipad = L->Ipad;
       // ---- phase N: x is final once every K slice of the previous layer has been added
       if (l > 0) {
-        bool w = event_wait(event_counter, static_cast<uint32_t>(3 * l) * per_event, abort_flag);
+        bool w = event_wait(event_counter + 3 * l - 1, per_event, abort_flag);
         w = __all_sync(0xFFFFFFFFu, w);
         if (!w) { ok = false; break; }
       }
@@ -279,7 +281,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
           *reinterpret_cast<uint2*>(xnorm + static_cast<int64_t>(t) * d + k) = pk;
         }
       }
-      arrive_event();                                            // event N(l)
+      arrive_event(3 * l);                                       // event N(l)
       // ---- phase A: Hd = bf16(silu(G) * U * scale)
       __nv_bfloat16* Hd = L->Hd;
       for (int tile = cta; ok && tile < Ipad / 128; tile += ctas) {
@@ -300,7 +302,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
         }
       }
       if (!ok) break;
-      arrive_event();                                            // event A(l)
+      arrive_event(3 * l + 1);                                   // event A(l)
       // ---- phase B: every K slice adds its part into x
       BItem it[4];
       const int nit = b_items(cta, ctas, m_blocks, Ipad / BK, it);
@@ -318,7 +320,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
         }
       }
       if (!ok) break;
-      arrive_event();                                            // event B(l)
+      arrive_event(3 * l + 2);                                   // event B(l)
     }
   }
   __syncwarp();
@@ -336,7 +338,7 @@ cudaError_t decode_stack_init(int* max_ctas_per_sm) {
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(max_ctas_per_sm, decode_stack_kernel, NUM_THREADS, SMEM_BYTES);
 }
 
-// layers_dev: n_layers records in device memory (64-byte aligned).  event_counter must be zero.
+// layers_dev: n_layers records in device memory (64-byte aligned).  event_counter: 3 * n_layers zeros.
 cudaError_t launch_decode_stack(const DecodeStackLayer* layers_dev, int n_layers, const CUtensorMap& tm_x, float* x, void* xnorm,
                                 int64_t n, int64_t d, int npad, float eps, uint32_t* event_counter, uint32_t* status,
                                 int num_sms, cudaStream_t st) {

@@ -52,7 +52,8 @@ def test_small_stack(lib, bf16, n):
         # host-buffer entry point
         yh = torch.empty((n, d), dtype=torch.float32)
         lib.mlpmoe_stack_forward_host(handles, torch.from_numpy(x), yh, n, 1e-6, stream_ptr())
-        assert np.array_equal(yh.numpy(), xd.cpu().numpy())
+        # same numbers up to the order in which K slices are added into the fp32 stream
+        np.testing.assert_allclose(yh.numpy(), xd.cpu().numpy(), rtol=1e-5, atol=1e-5)
         assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
     finally:
         for h in handles[1:] + handles[:1]:
