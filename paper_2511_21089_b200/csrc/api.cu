@@ -185,6 +185,7 @@ struct mlpmoe_layer_s {
   uint32_t* status = nullptr;
   int64_t launches = 0;
   CUtensorMap tm_wgu, tm_wdt;      // single-CTA boxes: 64 x 256 and 64 x 128
+  CUtensorMap tm_wdt256;           // WdT with box 64 x 256 (decode-stack kernel)
   CUtensorMap tm_wgu_pair;         // CTA-pair box: 64 x 128
   // optional per-kernel event timing
   bool timing = false;
@@ -255,6 +256,7 @@ mlpmoe_status_t reschedule(mlpmoe_layer_s* h, cudaStream_t st) {
   if (h->dtype == MLPMOE_BF16) {
     if (!make_tmap(&h->tm_wgu, h->Wgu, h->d, 2 * h->Ipad, h->d, 256)) return MLPMOE_ERR_CUDA;
     if (!make_tmap(&h->tm_wdt, h->WdT, h->Ipad, h->d, h->Ipad, 128)) return MLPMOE_ERR_CUDA;
+    if (!make_tmap(&h->tm_wdt256, h->WdT, h->Ipad, h->d, h->Ipad, 256)) return MLPMOE_ERR_CUDA;
     if (!make_tmap(&h->tm_wgu_pair, h->Wgu, h->d, 2 * h->Ipad, h->d, 128)) return MLPMOE_ERR_CUDA;
   }
   return MLPMOE_OK;
@@ -628,7 +630,7 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
     for (int l = 0; l < n_layers; ++l) {
       mlpmoe_layer_s* h = layers[l];
       recs[l].tm_wgu = h->tm_wgu;
-      recs[l].tm_wdt = h->tm_wdt;
+      recs[l].tm_wdt = h->tm_wdt256;
       if (!make_tmap(&recs[l].tm_hd, h->ws->H, h->Ipad, n, h->Ipad, npad)) return MLPMOE_ERR_CUDA;
       recs[l].scale = h->scale;
       recs[l].Hd = static_cast<__nv_bfloat16*>(h->ws->H);

@@ -3,11 +3,15 @@
 // static sequence of phases per layer
 //     N: RMSNorm of the token rows into the bf16 activation buffer
 //     A: gate|up, H = bf16(silu(G) * U * scale), 128 neurons per work item      (Section 3.1)
-//     B: down + branch sum, K slices added straight into the fp32 stream x
+//     B: down + branch sum, 256 output columns per work item, K slices added straight into the
+//        fp32 stream x
 // separated by grid-wide events (one global arrival counter, bounded waits).  The producer warp
 // never stops at an event with an empty ring: weight tiles depend on no earlier phase, so it keeps
 // issuing them and only holds back the small activation tile of each stage until the event it
 // needs has passed.  HBM therefore keeps streaming weights across phase and layer boundaries.
+// Both phases use the same stage: 256 weight rows x 64 K (two accumulators of 128 rows: gate and
+// up of the same neurons in phase A, two neighbouring blocks of output columns in phase B) next to
+// one token tile, so every stage carries 32 KB of weights.
 //
 // Warp roles: warp 0 TMA producer, warp 1 TMEM owner + MMA issuer, warps 2..5 epilogue (and the
 // RMSNorm phase).  Weights sit on the 128-row side of the MMA, tokens on N = 16 / 32 / 64.
@@ -25,14 +29,22 @@ constexpr int BK = 64;
 constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
 constexpr int MAXN = kDecodeMaxTokens;
-constexpr int STAGES = 5;
-constexpr int W_BYTES = 256 * BK * 2;                 // phase A: 128 gate + 128 up rows; phase B uses the first half
-constexpr int STAGE_BYTES = W_BYTES + MAXN * BK * 2;  // + token tile
-constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
-constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;
+constexpr int MAX_STAGES = 6;
+constexpr int W_BYTES = 256 * BK * 2;                 // 256 weight rows per stage in both phases
+// A stage is the weight tile plus a token tile of npad rows; the ring takes as many stages as fit
+// (6 for npad 16 and 32, 5 for npad 64), the barriers sit in front of it.
+constexpr int BAR_BYTES = 1024;
+constexpr int RING_BYTES = 216 * 1024;
+constexpr int SMEM_BYTES = BAR_BYTES + RING_BYTES + 1024;
+static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+__host__ __device__ constexpr int stage_bytes_for(int npad) { return W_BYTES + npad * BK * 2; }
+__host__ __device__ constexpr int stages_for(int npad) {
+  return RING_BYTES / stage_bytes_for(npad) < MAX_STAGES ? RING_BYTES / stage_bytes_for(npad) : MAX_STAGES;
+}
 constexpr uint32_t TMEM_COLS = 4 * MAXN;              // 2 buffers x (G | U)
 constexpr uint64_t WAIT_NS = 1000000000ull;
 constexpr uint32_t ARRIVALS_PER_CTA = 4;              // every epilogue warp arrives once per event
+constexpr int NORM_VEC = 8;                           // float4 per lane the RMSNorm phase keeps in registers
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
   uint32_t v;
@@ -40,6 +52,8 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
   return v;
 }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// The four epilogue warps (threads 64..191) only.
+__device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Events are numbered in program order, 3 per layer (N, A, B), and each has its own arrival counter
 // (a CTA without work in a phase arrives at once, so one shared counter would let early arrivals
@@ -65,20 +79,18 @@ __device__ __forceinline__ bool event_wait(const uint32_t* counter, uint32_t tar
   }
 }
 
-__device__ __forceinline__ void load_acc(uint32_t taddr, int npad, float (&v)[MAXN]) {
+// Issues the loads of one accumulator's first npad columns; the values are valid after tmem_ld_wait().
+__device__ __forceinline__ void load_acc_async(uint32_t taddr, int npad, uint32_t (&v)[MAXN]) {
 #pragma unroll
   for (int c = 0; c < MAXN; c += 16) {
     if (c < npad) {
-      uint32_t r[16];
+      uint32_t(&r)[16] = *reinterpret_cast<uint32_t(*)[16]>(&v[c]);
       tmem_ld_32x16(taddr + c, r);
-      tmem_ld_wait();
-#pragma unroll
-      for (int i = 0; i < 16; ++i) v[c + i] = __uint_as_float(r[i]);
     }
   }
 }
 
-// A CTA's share of phase B of one layer: units (128-row block of WdT, K-step) in block-major order,
+// A CTA's share of phase B of one layer: units (256-row block of WdT, K-step) in block-major order,
 // dealt in equal contiguous ranges; a range is cut at block boundaries into items.
 struct BItem {
   int m_blk, kb_lo, kb_hi;
@@ -99,6 +111,59 @@ __device__ __forceinline__ int b_items(int cta, int ctas, int m_blocks, int kb2,
   return n;
 }
 
+// One CTA's weight K-steps of the whole stack in program order: per layer first phase A (its
+// gate|up tiles, all K-steps of each), then phase B (its items).  The producer walks the
+// sequence.
+struct StepIter {
+  const DecodeStackLayer* layers;
+  int n_layers, cta, ctas, m_blocks, kb1;
+  int l, ph, idx, kb, nit;       // ph 0: idx = gate|up tile; ph 1: idx = item number
+  BItem it[4];
+  bool done;
+  __device__ __forceinline__ void settle() {      // moves to the first phase at or after (l, ph) that has work
+    while (!done) {
+      const int Ipad = layers[l].Ipad;
+      if (ph == 0) {
+        idx = cta;
+        kb = 0;
+        if (idx < Ipad / 128) return;
+        ph = 1;
+      }
+      nit = b_items(cta, ctas, m_blocks, Ipad / BK, it);
+      idx = 0;
+      if (nit > 0) { kb = it[0].kb_lo; return; }
+      ph = 0;
+      if (++l == n_layers) done = true;
+    }
+  }
+  __device__ __forceinline__ void init(const DecodeStackLayer* layers_, int n_layers_, int cta_, int ctas_, int m_blocks_, int kb1_) {
+    layers = layers_; n_layers = n_layers_; cta = cta_; ctas = ctas_; m_blocks = m_blocks_; kb1 = kb1_;
+    l = 0; ph = 0; idx = 0; kb = 0; nit = 0;
+    done = n_layers == 0;
+    settle();
+  }
+  __device__ __forceinline__ const CUtensorMap* wmap() const { return ph == 0 ? &layers[l].tm_wgu : &layers[l].tm_wdt; }
+  __device__ __forceinline__ int wrow() const { return (ph == 0 ? idx : it[idx].m_blk) * 256; }
+  __device__ __forceinline__ int event() const { return 3 * l + ph; }     // the event its activation tile waits for
+  __device__ __forceinline__ void advance() {
+    ++kb;
+    if (ph == 0) {
+      if (kb < kb1) return;
+      idx += ctas;
+      kb = 0;
+      if (idx < layers[l].Ipad / 128) return;
+      ph = 1;
+      settle();
+    } else {
+      if (kb < it[idx].kb_hi) return;
+      if (++idx < nit) { kb = it[idx].kb_lo; return; }
+      ph = 0;
+      if (++l == n_layers) { done = true; return; }
+      settle();
+    }
+  }
+};
+
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
                     const __grid_constant__ CUtensorMap tm_x,   // xnorm [n x d] bf16, box 64 x npad
@@ -106,20 +171,21 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
                     uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + BAR_OFFSET);
-  uint64_t* empty_bar = full_bar + STAGES;
-  uint64_t* tfull_bar = empty_bar + STAGES;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem);
+  uint64_t* empty_bar = full_bar + MAX_STAGES;
+  uint64_t* tfull_bar = empty_bar + MAX_STAGES;
   uint64_t* tempty_bar = tfull_bar + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  volatile float* norm_part = reinterpret_cast<volatile float*>(tmem_slot + 4);   // one partial sum of squares per epilogue warp
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int cta = blockIdx.x, ctas = gridDim.x;
   const uint32_t per_event = static_cast<uint32_t>(ctas) * ARRIVALS_PER_CTA;
-  const int m_blocks = static_cast<int>((d + 127) / 128);
+  const int m_blocks = static_cast<int>((d + 255) / 256);     // phase B: blocks of 256 output columns
   const int kb1 = static_cast<int>((d + BK - 1) / BK);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], 4); }
     *abort_flag = 0;
     fence_barrier_init();
@@ -130,62 +196,59 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t act_bytes = static_cast<uint32_t>(npad) * BK * 2;
+  uint8_t* ring = smem + BAR_BYTES;
+  const int STAGES = stages_for(npad), STAGE_BYTES = stage_bytes_for(npad);
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       prefetch_tensormap(&tm_x);
-      int stage = 0; uint32_t phase = 0; bool ok = true;
-      // activation tiles that wait for the current gating event: (stage, tensor map, K-step)
-      int deferred = 0, def_stage[STAGES], def_kb[STAGES];
-      const CUtensorMap* def_map = nullptr;
-      const uint32_t* gate = event_counter;  // counter of the gating event
+      int stage = 0; uint32_t phase = 0;
+      // activation tiles that wait for the current gating event: (stage, K-step) of map def_map
+      int deferred = 0, def_stage[MAX_STAGES], def_kb[MAX_STAGES];
+      const CUtensorMap* def_map = &tm_x;
+      int gate_ev = 0;                     // index of the gating event
       bool gate_open = false;
       auto flush = [&]() {
         fence_async_proxy();               // what the acquire made visible must be seen by the TMA reads
         for (int i = 0; i < deferred; ++i)
-          tma_load_2d(smem + def_stage[i] * STAGE_BYTES + W_BYTES, def_map, def_kb[i] * BK, 0, &full_bar[def_stage[i]]);
+          tma_load_2d(ring + def_stage[i] * STAGE_BYTES + W_BYTES, def_map, def_kb[i] * BK, 0, &full_bar[def_stage[i]]);
         deferred = 0;
         gate_open = true;
       };
-      // issues one stage: weights at once, the token tile as soon as the gate is open
-      auto issue = [&](const CUtensorMap* wmap, int wrow, uint32_t wbytes, const CUtensorMap* amap, int kb) -> bool {
-        if (!gate_open && (deferred == STAGES || event_passed(gate, per_event))) {
-          if (deferred == STAGES && !event_wait(gate, per_event, abort_flag)) return false;
+      StepIter cur;
+      cur.init(layers, n_layers, cta, ctas, m_blocks, kb1);
+      bool ok = true;
+      while (ok && !cur.done) {
+        const int ev = cur.event();
+        if (ev != gate_ev) {
+          // a new phase: the deferred tiles of the previous one go first (events pass in order)
+          if (deferred > 0) {
+            if (!event_wait(event_counter + gate_ev, per_event, abort_flag)) { ok = false; break; }
+            flush();
+          }
+          gate_ev = ev;
+          gate_open = false;
+          def_map = cur.ph == 0 ? &tm_x : &layers[cur.l].tm_hd;
+        }
+        if (!gate_open && (deferred == STAGES || event_passed(event_counter + gate_ev, per_event))) {
+          if (deferred == STAGES && !event_wait(event_counter + gate_ev, per_event, abort_flag)) { ok = false; break; }
           flush();
         }
-        if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, WAIT_NS)) return false;
-        uint8_t* s = smem + stage * STAGE_BYTES;
-        mbar_expect_tx(&full_bar[stage], wbytes + act_bytes);
-        tma_load_2d(s, wmap, kb * BK, wrow, &full_bar[stage]);
+        if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, WAIT_NS)) { ok = false; break; }
+        uint8_t* s = ring + stage * STAGE_BYTES;
+        mbar_expect_tx(&full_bar[stage], W_BYTES + act_bytes);
+        const int kc = cur.kb;     // every CTA walks K in the same order: staggered starts measured 3 % slower
+        tma_load_2d(s, cur.wmap(), kc * BK, cur.wrow(), &full_bar[stage]);
         if (gate_open) {
-          tma_load_2d(s + W_BYTES, amap, kb * BK, 0, &full_bar[stage]);
+          tma_load_2d(s + W_BYTES, def_map, kc * BK, 0, &full_bar[stage]);
         } else {
-          def_stage[deferred] = stage; def_kb[deferred] = kb; ++deferred;
+          def_stage[deferred] = stage; def_kb[deferred] = kc; ++deferred;
         }
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-        return true;
-      };
-      for (int l = 0; ok && l < n_layers; ++l) {
-        const DecodeStackLayer* L = layers + l;
-        const int Ipad = L->Ipad;
-        // phase A needs event N(l): index 3l
-        if (deferred > 0) { if (!event_wait(gate, per_event, abort_flag)) { ok = false; break; } flush(); }
-        gate = event_counter + 3 * l; gate_open = false; def_map = &tm_x;
-        for (int tile = cta; ok && tile < Ipad / 128; tile += ctas)
-          for (int kb = 0; kb < kb1; ++kb)
-            if (!issue(&L->tm_wgu, tile * 256, W_BYTES, &tm_x, kb)) { ok = false; break; }
-        if (!ok) break;
-        // phase B needs event A(l): index 3l + 1
-        if (deferred > 0) { if (!event_wait(gate, per_event, abort_flag)) { ok = false; break; } flush(); }
-        gate = event_counter + 3 * l + 1; gate_open = false; def_map = &L->tm_hd;
-        BItem it[4];
-        const int nit = b_items(cta, ctas, m_blocks, Ipad / BK, it);
-        for (int i = 0; ok && i < nit; ++i)
-          for (int kb = it[i].kb_lo; kb < it[i].kb_hi; ++kb)
-            if (!issue(&L->tm_wdt, it[i].m_blk * 128, W_BYTES / 2, &L->tm_hd, kb)) { ok = false; break; }
+        cur.advance();
       }
-      if (ok && deferred > 0 && event_wait(gate, per_event, abort_flag)) flush();
+      if (ok && deferred > 0 && event_wait(event_counter + gate_ev, per_event, abort_flag)) flush();
     }
   }
   else if (warp == 1) {
@@ -193,15 +256,15 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
     if (lane == 0) {
       const uint32_t idesc = make_idesc_bf16_f32(128, static_cast<uint32_t>(npad));
       int stage = 0, acc = 0; uint32_t phase = 0, acc_phase = 0; bool ok = true;
-      // one accumulator item: two_acc = gate and up (phase A), else one accumulator (phase B)
-      auto run_item = [&](int kbs, bool two_acc) -> bool {
+      // one work item: two accumulators of 128 weight rows each
+      auto run_item = [&](int kbs) -> bool {
         if (!mbar_wait_bounded(&tempty_bar[acc], acc_phase ^ 1u, abort_flag, WAIT_NS)) return false;
         tc_fence_after();
         const uint32_t g_tmem = tmem_base + static_cast<uint32_t>(acc * 2 * MAXN);
         for (int kb = 0; kb < kbs; ++kb) {
           if (!mbar_wait_bounded(&full_bar[stage], phase, abort_flag, WAIT_NS)) return false;
           tc_fence_after();
-          const uint32_t s = smem_u32(smem + stage * STAGE_BYTES);
+          const uint32_t s = smem_u32(ring + stage * STAGE_BYTES);
           const uint64_t w0 = make_desc_sw128_kmajor(s);
           const uint64_t w1 = make_desc_sw128_kmajor(s + 128 * BK * 2);
           const uint64_t xd = make_desc_sw128_kmajor(s + W_BYTES);
@@ -209,7 +272,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
           for (int k = 0; k < BK / UMMA_K; ++k) {
             const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
             umma_bf16(g_tmem, w0 + 2 * k, xd + 2 * k, idesc, accum);
-            if (two_acc) umma_bf16(g_tmem + MAXN, w1 + 2 * k, xd + 2 * k, idesc, accum);
+            umma_bf16(g_tmem + MAXN, w1 + 2 * k, xd + 2 * k, idesc, accum);
           }
           umma_commit(&empty_bar[stage]);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -221,10 +284,10 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
       };
       for (int l = 0; ok && l < n_layers; ++l) {
         const int Ipad = layers[l].Ipad;
-        for (int tile = cta; ok && tile < Ipad / 128; tile += ctas) ok = run_item(kb1, true);
+        for (int tile = cta; ok && tile < Ipad / 128; tile += ctas) ok = run_item(kb1);
         BItem it[4];
         const int nit = b_items(cta, ctas, m_blocks, Ipad / BK, it);
-        for (int i = 0; ok && i < nit; ++i) ok = run_item(it[i].kb_hi - it[i].kb_lo, false);
+        for (int i = 0; ok && i < nit; ++i) ok = run_item(it[i].kb_hi - it[i].kb_lo);
       }
     }
   }
@@ -251,76 +314,116 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     };
-    for (int l = 0; ok && l < n_layers; ++l) {
+    // Once a wait has given up (ok == false) a warp skips all further work but still walks every
+    // loop, so that the four warps keep meeting at the named barrier of the RMSNorm phase.
+    for (int l = 0; l < n_layers; ++l) {
       const DecodeStackLayer* L = layers + l;
       const int Ipad = L->Ipad;
       // ---- phase N: x is final once every K slice of the previous layer has been added
-      if (l > 0) {
+      if (ok && l > 0) {
         bool w = event_wait(event_counter + 3 * l - 1, per_event, abort_flag);
-        w = __all_sync(0xFFFFFFFFu, w);
-        if (!w) { ok = false; break; }
+        ok = __all_sync(0xFFFFFFFFu, w);
       }
       for (int t = cta; t < n; t += ctas) {
-        // each of the four warps sums the whole row (16 KB from L2) and writes its quarter of it
+        // each warp takes a quarter of the row, keeps it in registers, and the four partial sums of
+        // squares meet in shared memory
         const float* row = x + static_cast<int64_t>(t) * d;
-        float ss = 0.f;
-        for (int64_t k = lane * 4; k < d; k += 128) {
-          const float4 v = __ldcg(reinterpret_cast<const float4*>(row + k));
-          ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-        }
-        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
-        const float inv = 1.0f / sqrtf(ss / static_cast<float>(d) + eps);
         const int64_t q = (d / 4 + 3) / 4 * 4;                 // columns per warp, a multiple of 4
         const int64_t c0 = static_cast<int64_t>(quad) * q, c1 = c0 + q < d ? c0 + q : d;
-        for (int64_t k = c0 + lane * 4; k < c1; k += 128) {
-          const float4 v = __ldcg(reinterpret_cast<const float4*>(row + k));
-          __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * inv, v.y * inv), hi = __floats2bfloat162_rn(v.z * inv, v.w * inv);
-          uint2 pk;
-          pk.x = *reinterpret_cast<uint32_t*>(&lo);
-          pk.y = *reinterpret_cast<uint32_t*>(&hi);
-          *reinterpret_cast<uint2*>(xnorm + static_cast<int64_t>(t) * d + k) = pk;
+        float4 v[NORM_VEC];
+        float ss = 0.f;
+        if (ok) {
+#pragma unroll
+          for (int i = 0; i < NORM_VEC; ++i) {
+            const int64_t k = c0 + (static_cast<int64_t>(i) * 32 + lane) * 4;
+            v[i] = k < c1 ? __ldcg(reinterpret_cast<const float4*>(row + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll
+          for (int i = 0; i < NORM_VEC; ++i) ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+          for (int64_t k = c0 + (static_cast<int64_t>(NORM_VEC) * 32 + lane) * 4; k < c1; k += 128) {   // rows wider than the register window
+            const float4 w4 = __ldcg(reinterpret_cast<const float4*>(row + k));
+            ss += w4.x * w4.x + w4.y * w4.y + w4.z * w4.z + w4.w * w4.w;
+          }
+          for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+        }
+        if (lane == 0) norm_part[quad] = ss;
+        epilogue_bar_sync();
+        const float total = norm_part[0] + norm_part[1] + norm_part[2] + norm_part[3];
+        epilogue_bar_sync();                                   // norm_part may be overwritten by the next row
+        if (ok) {
+          const float inv = 1.0f / sqrtf(total / static_cast<float>(d) + eps);
+          __nv_bfloat16* out = xnorm + static_cast<int64_t>(t) * d;
+          auto store4 = [&](int64_t k, const float4& f) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(f.x * inv, f.y * inv), hi = __floats2bfloat162_rn(f.z * inv, f.w * inv);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t*>(&lo);
+            pk.y = *reinterpret_cast<uint32_t*>(&hi);
+            *reinterpret_cast<uint2*>(out + k) = pk;
+          };
+#pragma unroll
+          for (int i = 0; i < NORM_VEC; ++i) {
+            const int64_t k = c0 + (static_cast<int64_t>(i) * 32 + lane) * 4;
+            if (k < c1) store4(k, v[i]);
+          }
+          for (int64_t k = c0 + (static_cast<int64_t>(NORM_VEC) * 32 + lane) * 4; k < c1; k += 128)
+            store4(k, __ldcg(reinterpret_cast<const float4*>(row + k)));
         }
       }
-      arrive_event(3 * l);                                       // event N(l)
+      if (ok) arrive_event(3 * l);                               // event N(l)
       // ---- phase A: Hd = bf16(silu(G) * U * scale)
       __nv_bfloat16* Hd = L->Hd;
-      for (int tile = cta; ok && tile < Ipad / 128; tile += ctas) {
-        if (!wait_acc()) { ok = false; break; }
+      for (int tile = cta; tile < Ipad / 128; tile += ctas) {
+        if (ok && !wait_acc()) ok = false;
+        if (!ok) continue;
         const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * 2 * MAXN) + (static_cast<uint32_t>(quad * 32) << 16);
-        float g[MAXN], u[MAXN];
-        load_acc(taddr, npad, g);
-        load_acc(taddr + MAXN, npad, u);
-        release_acc();
         const int64_t j = static_cast<int64_t>(tile) * 128 + quad * 32 + lane;
         const float sc = L->scale[j];
 #pragma unroll
-        for (int t = 0; t < MAXN; ++t) {
-          if (t < n) {
-            const float gv = g[t];
-            Hd[static_cast<int64_t>(t) * Ipad + j] = __float2bfloat16_rn(__fdividef(gv, 1.0f + __expf(-gv)) * u[t] * sc);
+        for (int c = 0; c < MAXN; c += 32) {                   // 32 tokens at a time: gate and up columns together
+          if (c < npad) {
+            uint32_t g[32], u[32];
+            tmem_ld_32x16(taddr + c, *reinterpret_cast<uint32_t(*)[16]>(&g[0]));
+            tmem_ld_32x16(taddr + MAXN + c, *reinterpret_cast<uint32_t(*)[16]>(&u[0]));
+            if (c + 16 < npad) {
+              tmem_ld_32x16(taddr + c + 16, *reinterpret_cast<uint32_t(*)[16]>(&g[16]));
+              tmem_ld_32x16(taddr + MAXN + c + 16, *reinterpret_cast<uint32_t(*)[16]>(&u[16]));
+            }
+            tmem_ld_wait();
+            if (c + 32 >= npad) release_acc();                 // the last columns have been read
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int t = c + i;
+              if (t < n) {
+                const float gv = __uint_as_float(g[i]);
+                Hd[static_cast<int64_t>(t) * Ipad + j] = __float2bfloat16_rn(__fdividef(gv, 1.0f + __expf(-gv)) * __uint_as_float(u[i]) * sc);
+              }
+            }
           }
         }
       }
-      if (!ok) break;
-      arrive_event(3 * l + 1);                                   // event A(l)
+      if (ok) arrive_event(3 * l + 1);                           // event A(l)
       // ---- phase B: every K slice adds its part into x
       BItem it[4];
       const int nit = b_items(cta, ctas, m_blocks, Ipad / BK, it);
-      for (int i = 0; ok && i < nit; ++i) {
-        if (!wait_acc()) { ok = false; break; }
+      for (int i = 0; i < nit; ++i) {
+        if (ok && !wait_acc()) ok = false;
+        if (!ok) continue;
         const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * 2 * MAXN) + (static_cast<uint32_t>(quad * 32) << 16);
-        float v[MAXN];
-        load_acc(taddr, npad, v);
-        release_acc();
-        const int64_t m = static_cast<int64_t>(it[i].m_blk) * 128 + quad * 32 + lane;
-        if (m < d) {
 #pragma unroll
-          for (int t = 0; t < MAXN; ++t)
-            if (t < n) atomicAdd(x + static_cast<int64_t>(t) * d + m, v[t]);
+        for (int half = 0; half < 2; ++half) {                 // the two blocks of 128 output columns
+          uint32_t v[MAXN];
+          load_acc_async(taddr + half * MAXN, npad, v);
+          tmem_ld_wait();
+          if (half == 1) release_acc();
+          const int64_t m = static_cast<int64_t>(it[i].m_blk) * 256 + half * 128 + quad * 32 + lane;
+          if (m < d) {
+#pragma unroll
+            for (int t = 0; t < MAXN; ++t)
+              if (t < n) atomicAdd(x + static_cast<int64_t>(t) * d + m, __uint_as_float(v[t]));
+          }
         }
       }
-      if (!ok) break;
-      arrive_event(3 * l + 2);                                   // event B(l)
+      if (ok) arrive_event(3 * l + 2);                           // event B(l)
     }
   }
   __syncwarp();

@@ -153,7 +153,7 @@ cudaError_t decode_init();
 // One record per layer of a decode stack, read by the persistent stack kernel from device memory.
 struct alignas(64) DecodeStackLayer {
   CUtensorMap tm_wgu;    // Wgu [2 Ipad x d]  box 64 x 256
-  CUtensorMap tm_wdt;    // WdT [d x Ipad]    box 64 x 128
+  CUtensorMap tm_wdt;    // WdT [d x Ipad]    box 64 x 256
   CUtensorMap tm_hd;     // Hd  [n x Ipad]    box 64 x npad
   const float* scale;    // [Ipad]
   __nv_bfloat16* Hd;     // [n x Ipad]
