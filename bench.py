@@ -91,7 +91,7 @@ def layer_inputs(layer: int, w):
 # profiles/tc_layer_kernel_qwen_c2_2layers.md (dram__bytes_read.sum + dram__bytes_write.sum), valid
 # only while the kernel's sources are the ones that were profiled.
 GATEUP_TRAFFIC_BYTES = 42.16e6 + 4.08e6
-GATEUP_SOURCES = ("tc_layer.cu", "tc_common.cuh", "ptx.cuh")
+GATEUP_SOURCES = ("tc_stack.cu", "tc_common.cuh", "ptx.cuh")
 GATEUP_SOURCES_SHA = "058b6e7cb57620d0"
 
 
@@ -385,14 +385,23 @@ def run_ours(args):
             "weight_gbs": weights_gb / (ms_step * 1e-3),
         }
         if kcnt[0] > 0:
+            # per-kernel events exist on every 8th step only: shares are taken of those steps' time
+            timed_steps = len(range(0, args.steps, 8))
+            ms_timed = ms_total * timed_steps / args.steps
             gu_ms = kms[0] / kcnt[0]
             dn_ms = kms[1] / max(kcnt[1], 1)
             fused = n > 128            # one kernel runs both GEMMs of a layer call
+            whole_stack = fused and w["stack"]     # ... and, for a stack, every layer and its RMSNorm
             if n > 64:
-                flops = float(np.mean(flops_gu)) + (float(np.mean(flops_dn)) if fused else 0.0)
+                if whole_stack:
+                    flops = float(np.sum(flops_gu)) + float(np.sum(flops_dn))
+                else:
+                    flops = float(np.mean(flops_gu)) + (float(np.mean(flops_dn)) if fused else 0.0)
                 achieved = flops / (gu_ms * 1e-3) / 1e12
                 out["roofline"] = {"bound": "tensor",
-                                   "kernel": "fused layer kernel: gate|up GEMM + SiLU*up epilogue, then down GEMM (tcgen05, CTA pairs)"
+                                   "kernel": "persistent stack kernel: per layer RMSNorm, gate|up GEMM + SiLU*up epilogue, down GEMM + "
+                                             "residual add (tcgen05, CTA pairs, all layers in one launch)" if whole_stack else
+                                   "fused layer kernel: gate|up GEMM + SiLU*up epilogue, then down GEMM (tcgen05, CTA pairs)"
                                    if fused else "gate|up GEMM + SiLU*up epilogue (tcgen05)",
                                    "achieved": achieved, "peak": pk["tflops_sustained"], "unit": "TFLOP/s",
                                    "frac": achieved / pk["tflops_sustained"], "traffic": gateup_traffic() if default else None,
@@ -404,21 +413,24 @@ def run_ours(args):
                                    "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
                                    "traffic": None, "peak_source": pk["source"] + " (copy bandwidth)", "avg_launch_us": gu_ms * 1e3}
             if n <= 64:
-                out["kernels"] = {"decode_stack": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_total),
+                out["kernels"] = {"decode_stack": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_timed),
                                                    "weight_gbs": achieved}}
+            elif whole_stack:
+                out["kernels"] = {"prefill_stack": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_timed),
+                                                    "tflops": achieved}}
             elif fused:
                 out["kernels"] = {
-                    "layer_fused": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_total),
+                    "layer_fused": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_timed),
                                     "tflops": achieved},
-                    "rmsnorm": {"avg_us": kms[2] / max(kcnt[2], 1) * 1e3, "launches": int(kcnt[2]), "share": float(kms[2] / ms_total)},
+                    "rmsnorm": {"avg_us": kms[2] / max(kcnt[2], 1) * 1e3, "launches": int(kcnt[2]), "share": float(kms[2] / ms_timed)},
                 }
             else:
                 out["kernels"] = {
-                "gate_up": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_total),
+                "gate_up": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_timed),
                             "tflops": float(np.mean(flops_gu)) / (gu_ms * 1e-3) / 1e12, "weight_gbs": float(np.mean(wbytes_gu)) / (gu_ms * 1e-3) / 1e9},
-                "down": {"avg_us": dn_ms * 1e3, "launches": int(kcnt[1]), "share": float(kms[1] / ms_total),
+                "down": {"avg_us": dn_ms * 1e3, "launches": int(kcnt[1]), "share": float(kms[1] / ms_timed),
                          "tflops": float(np.mean(flops_dn)) / (dn_ms * 1e-3) / 1e12, "weight_gbs": float(np.mean(wbytes_dn)) / (dn_ms * 1e-3) / 1e9},
-                "rmsnorm": {"avg_us": kms[2] / max(kcnt[2], 1) * 1e3, "launches": int(kcnt[2]), "share": float(kms[2] / ms_total)},
+                "rmsnorm": {"avg_us": kms[2] / max(kcnt[2], 1) * 1e3, "launches": int(kcnt[2]), "share": float(kms[2] / ms_timed)},
             }
         else:
             out["roofline"] = None

@@ -276,6 +276,23 @@ mlpmoe_status_t mlpmoe_host_tile_schedule(int64_t n_tokens, int64_t d_model, int
                                           int32_t ksplit, int32_t num_sms, int32_t* tiles, int32_t* n_tiles,
                                           int32_t* offsets);
 
+/*
+ * The work sequences of the persistent prefill-stack kernel (mlpmoe_stack_forward with more than
+ * 128 tokens): which CTA pair runs which items of which layer in which order (set-up logic, no
+ * CUDA call).  Every pair has two independent sequences: its GEMM items (per layer and 256-token
+ * block n_active_pad[l]/128 gate|up tiles and ksplit[l] * ceil(d_model/bn) down items) and the norm
+ * parts (16 per layer and block, 16 token rows each) that its norm warps run.  items:
+ * item_capacity pairs of int32 (code, layer), code = type << 30 | column << 16 | token block with
+ * type 0 = gate|up tile, 1 = down item (column = column tile * ksplit + slice), 2 = norm part
+ * (column = part); the GEMM sequences of all pairs come first, then the norm sequences.  *n_items
+ * receives the number of items (also when item_capacity is too small, which returns
+ * MLPMOE_ERR_INVALID_ARG); offsets: capacity 2 * (num_sms/2 + 1), in items: num_sms/2 + 1 bounds
+ * of the GEMM sequences, then num_sms/2 + 1 bounds of the norm sequences.
+ */
+mlpmoe_status_t mlpmoe_host_stack_schedule(int64_t n_tokens, int64_t d_model, int32_t n_layers, const int64_t* n_active_pad,
+                                           const int32_t* ksplit, int32_t bn, int32_t num_sms, int32_t* items,
+                                           int64_t item_capacity, int64_t* n_items, int32_t* offsets);
+
 #ifdef __cplusplus
 }
 #endif

@@ -63,6 +63,8 @@ SIGNATURES = {
     "mlpmoe_host_prune_alpha": (c_int32, [c_int32, POINTER(c_float), POINTER(c_uint8), c_int32, POINTER(c_float)]),
     "mlpmoe_host_tile_schedule": (c_int32, [c_int64, c_int64, c_int64, c_int32, c_int32, c_int32, POINTER(c_int32), POINTER(c_int32),
                                             POINTER(c_int32)]),
+    "mlpmoe_host_stack_schedule": (c_int32, [c_int64, c_int64, c_int32, POINTER(c_int64), POINTER(c_int32), c_int32, c_int32,
+                                             POINTER(c_int32), c_int64, POINTER(c_int64), POINTER(c_int32)]),
     "mlpmoe_host_schedule": (c_int32, [c_int32, POINTER(c_int64), POINTER(c_float), POINTER(c_uint8), POINTER(c_int32),
                                        POINTER(c_int32), POINTER(c_int64), POINTER(c_int64), POINTER(c_int32),
                                        POINTER(c_int64)]),
@@ -291,3 +293,24 @@ def mlpmoe_host_tile_schedule(n_tokens: int, d_model: int, n_active_pad: int, bn
     for c in range(num_sms // 2):
         out.append([((t >> 31) & 1, (t >> 16) & 0x7FFF, t & 0xFFFF) for t in tiles[offs[c]:offs[c + 1]]])
     return out
+
+
+def mlpmoe_host_stack_schedule(n_tokens: int, d_model: int, n_active_pad: Sequence[int], ksplit: Sequence[int], bn: int,
+                               num_sms: int = 148):
+    """Returns (gemm, norm): for each CTA pair its sequence of GEMM items and its sequence of norm
+    parts, as (type, column, token_block, layer); type 0 = gate|up tile, 1 = down item, 2 = norm part."""
+    L = len(n_active_pad)
+    m_pairs = (n_tokens + 255) // 256
+    pairs = num_sms // 2
+    cap = sum(m_pairs * (16 + ip // 128 + ks * ((d_model + bn - 1) // bn)) for ip, ks in zip(n_active_pad, ksplit))
+    items = (c_int32 * (2 * cap))()
+    n_items = c_int64()
+    offs = (c_int32 * (2 * (pairs + 1)))()
+    _check(lib.mlpmoe_host_stack_schedule(n_tokens, d_model, L, (c_int64 * L)(*n_active_pad), (c_int32 * L)(*ksplit), bn, num_sms,
+                                          items, cap, ctypes.byref(n_items), offs), "mlpmoe_host_stack_schedule")
+
+    def seq(lo, hi):
+        return [((items[2 * i] >> 30) & 3, (items[2 * i] >> 16) & 0x3FFF, items[2 * i] & 0xFFFF, items[2 * i + 1]) for i in range(lo, hi)]
+    gemm = [seq(offs[c], offs[c + 1]) for c in range(pairs)]
+    norm = [seq(offs[pairs + 1 + c], offs[pairs + 2 + c]) for c in range(pairs)]
+    return gemm, norm

@@ -174,6 +174,15 @@ struct mlpmoe_layer_s {
   DecodeStackLayer* stack_dev = nullptr;                    // layer records of the persistent decode-stack kernel
   uint32_t* stack_counter = nullptr;                        // its grid-wide event counter
   std::vector<DecodeStackLayer> stack_host;                 // what stack_dev currently holds
+  // persistent prefill-stack kernel (buffers live in the first layer's handle, sized at the first call
+  // with a new stack / token count)
+  TcStackLayer* pstack_dev = nullptr;
+  int32_t* pstack_items = nullptr;                          // work items, then the per-pair offsets
+  uint32_t* pstack_counters = nullptr;
+  int64_t pstack_layer_cap = 0, pstack_item_cap = 0, pstack_counter_cap = 0, pstack_n_items = 0;
+  int pstack_bn = 0;
+  std::vector<int64_t> pstack_key;                          // what the device buffers were built for
+  int64_t version = 0;                                      // bumped by every reschedule
   uint32_t* counters = nullptr;
   uint32_t* block_done = nullptr;                           // [2 x ceil(max_tokens / 256)] gate|up completion counters
   int64_t max_blocks = 0;
@@ -218,6 +227,7 @@ void free_layer(mlpmoe_layer_s* h) {
   cudaFree(h->Wgu); cudaFree(h->WdT);
   cudaFree(h->scale); cudaFree(h->src_row); cudaFree(h->row_nnz);
   cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->block_done); cudaFree(h->tile_sched); cudaFree(h->stack_dev); cudaFree(h->stack_counter); cudaFree(h->status);
+  cudaFree(h->pstack_dev); cudaFree(h->pstack_items); cudaFree(h->pstack_counters);
   ws_release(h->ws);
   delete h;
 }
@@ -225,6 +235,7 @@ void free_layer(mlpmoe_layer_s* h) {
 // Recompute liveness, the K-list, the per-neuron scale and the packed operands from the
 // canonical weights and the effective gates.  Synchronises `st`.
 mlpmoe_status_t reschedule(mlpmoe_layer_s* h, cudaStream_t st) {
+  h->version += 1;
   CK(launch_row_nnz(h->Wg_c, h->Wu_c, h->Wd_c, h->row_nnz, h->I, h->d, h->elem_size, st));
   h->row_nnz_host.resize(3 * h->I);
   CK(cudaMemcpyAsync(h->row_nnz_host.data(), h->row_nnz, sizeof(int32_t) * 3 * h->I, cudaMemcpyDeviceToHost, st));
@@ -413,6 +424,92 @@ mlpmoe_status_t check_stack(const mlpmoe_handle_t* layers, int32_t n_layers, int
   return MLPMOE_OK;
 }
 
+// Prefill of a stack whose layers share one workspace: the whole stack in one persistent CTA-pair
+// kernel.  The first call with a new stack, token count or schedule builds the work sequences on
+// the host and (re)sizes the device buffers that hold them; later calls only zero the counters
+// and launch.
+mlpmoe_status_t prefill_stack(const mlpmoe_handle_t* layers, int32_t n_layers, float* x, int64_t n, float eps, cudaStream_t st) {
+  mlpmoe_layer_s* h0 = layers[0];
+  const int64_t d = h0->d;
+  const int bn = tc_layer_down_bn(n, d, h0->num_sms);
+  const int64_t m_pairs = (n + 255) / 256;
+  std::vector<int64_t> key;
+  key.reserve(4 + 2 * static_cast<size_t>(n_layers));
+  key.push_back(n);
+  key.push_back(bn);
+  key.push_back(reinterpret_cast<int64_t>(h0->ws->H));
+  key.push_back(reinterpret_cast<int64_t>(h0->ws->xnorm));
+  for (int l = 0; l < n_layers; ++l) {
+    key.push_back(reinterpret_cast<int64_t>(layers[l]));
+    key.push_back(layers[l]->version);
+  }
+  if (key != h0->pstack_key) {
+    std::vector<TcStackLayer> recs(static_cast<size_t>(n_layers));
+    std::memset(recs.data(), 0, sizeof(TcStackLayer) * recs.size());
+    std::vector<int64_t> Ipad(n_layers);
+    std::vector<int> ksplit(n_layers);
+    for (int l = 0; l < n_layers; ++l) {
+      mlpmoe_layer_s* h = layers[l];
+      Ipad[l] = h->Ipad;
+      ksplit[l] = tc_layer_ksplit(n, d, h->Ipad, bn, TcLayerArgs::OUT_TMA_ADD, h0->num_sms);
+      recs[l].tm_wgu = h->tm_wgu_pair;
+      if (!make_tmap(&recs[l].tm_h_st, h->ws->H, h->Ipad, n, h->Ipad, 32)) return MLPMOE_ERR_CUDA;
+      if (!make_tmap(&recs[l].tm_h_ld, h->ws->H, h->Ipad, n, h->Ipad, 128)) return MLPMOE_ERR_CUDA;
+      if (!make_tmap(&recs[l].tm_wdt, h->WdT, h->Ipad, d, h->Ipad, bn / 2)) return MLPMOE_ERR_CUDA;
+      recs[l].scale = h->scale;
+      recs[l].n1 = static_cast<int32_t>(h->Ipad / 128);
+      recs[l].kb2 = static_cast<int32_t>(h->Ipad / 64);
+      recs[l].ksplit = ksplit[l];
+    }
+    std::vector<int32_t> items, offs;
+    tc_stack_schedule(n, d, Ipad.data(), ksplit.data(), n_layers, bn, h0->num_sms, &items, &offs);
+    const int64_t need_items = static_cast<int64_t>(items.size() + offs.size());
+    const int64_t need_counters = 3 * static_cast<int64_t>(n_layers) * m_pairs;
+    if (need_items > h0->pstack_item_cap || need_counters > h0->pstack_counter_cap || n_layers > h0->pstack_layer_cap) {
+      CK(cudaStreamSynchronize(st));     // earlier launches may still read the old buffers
+      cudaFree(h0->pstack_items); cudaFree(h0->pstack_counters); cudaFree(h0->pstack_dev);
+      h0->pstack_items = nullptr; h0->pstack_counters = nullptr; h0->pstack_dev = nullptr;
+      h0->pstack_item_cap = h0->pstack_counter_cap = h0->pstack_layer_cap = 0;
+      h0->pstack_key.clear();
+      if (cudaMalloc(reinterpret_cast<void**>(&h0->pstack_items), sizeof(int32_t) * need_items) != cudaSuccess ||
+          cudaMalloc(reinterpret_cast<void**>(&h0->pstack_counters), sizeof(uint32_t) * need_counters) != cudaSuccess ||
+          cudaMalloc(reinterpret_cast<void**>(&h0->pstack_dev), sizeof(TcStackLayer) * n_layers) != cudaSuccess)
+        return MLPMOE_ERR_ALLOC;
+      h0->pstack_item_cap = need_items; h0->pstack_counter_cap = need_counters; h0->pstack_layer_cap = n_layers;
+    }
+    items.insert(items.end(), offs.begin(), offs.end());
+    h0->pstack_n_items = static_cast<int64_t>(items.size() - offs.size());
+    CK(cudaMemcpyAsync(h0->pstack_items, items.data(), sizeof(int32_t) * items.size(), cudaMemcpyHostToDevice, st));
+    CK(cudaMemcpyAsync(h0->pstack_dev, recs.data(), sizeof(TcStackLayer) * recs.size(), cudaMemcpyHostToDevice, st));
+    CK(cudaStreamSynchronize(st));       // the host vectors above go out of scope
+    h0->pstack_key = key;
+    h0->pstack_bn = bn;
+  }
+  TcStackArgs a;
+  a.layers = h0->pstack_dev;
+  a.n_layers = n_layers;
+  if (!make_tmap(&a.tm_x, h0->ws->xnorm, d, n, d, 128)) return MLPMOE_ERR_CUDA;
+  if (!make_tmap_t(&a.tm_y, x, d, n, d, 32, 4)) return MLPMOE_ERR_CUDA;
+  a.x = x;
+  a.xnorm = h0->ws->xnorm;
+  a.n = n;
+  a.d = d;
+  a.bn = bn;
+  a.eps = eps;
+  a.items = h0->pstack_items;
+  a.list_offsets = h0->pstack_items + h0->pstack_n_items;
+  a.counters = h0->pstack_counters;
+  a.status = h0->status;
+  pdl_overlap_enabled() = !h0->timing;
+  CK(cudaMemsetAsync(h0->pstack_counters, 0, sizeof(uint32_t) * 3 * n_layers * m_pairs, st));
+  const long e0 = rec_event(h0, st);
+  CK(launch_tc_stack(a, h0->num_sms, st));
+  const long e1 = rec_event(h0, st);
+  add_span(h0, SPAN_GATEUP, e0, e1);       // the one kernel of the step is reported in the first slot
+  h0->launches += 1;
+  return MLPMOE_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -438,6 +535,7 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
   if (prop.major != 10) return MLPMOE_ERR_UNSUPPORTED;     // kernels are built for sm_100a only
   CK(tc_gemm_init());
   CK(tc_layer_init());
+  CK(tc_stack_init());
   CK(decode_init());
 
   mlpmoe_layer_s* h = new (std::nothrow) mlpmoe_layer_s();
@@ -652,6 +750,11 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
     h0->launches += 1;
     return MLPMOE_OK;
   }
+  if (layers[0]->dtype == MLPMOE_BF16 && n > 128 && n_layers <= kMaxStackLayers) {
+    bool same_ws = true;
+    for (int l = 1; l < n_layers; ++l) same_ws = same_ws && layers[l]->ws == layers[0]->ws;
+    if (same_ws) return prefill_stack(layers, n_layers, x, n, eps, st);
+  }
   for (int l = 0; l < n_layers; ++l) {
     mlpmoe_layer_s* h = layers[l];
     pdl_overlap_enabled() = !h->timing;
@@ -842,6 +945,24 @@ mlpmoe_status_t mlpmoe_host_tile_schedule(int64_t n_tokens, int64_t d_model, int
   std::memcpy(tiles, t.data(), sizeof(int32_t) * t.size());
   std::memcpy(offsets, o.data(), sizeof(int32_t) * o.size());
   *n_tiles = static_cast<int32_t>(t.size());
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_host_stack_schedule(int64_t n_tokens, int64_t d_model, int32_t n_layers, const int64_t* n_active_pad,
+                                           const int32_t* ksplit, int32_t bn, int32_t num_sms, int32_t* items,
+                                           int64_t item_capacity, int64_t* n_items, int32_t* offsets) {
+  if (n_tokens <= 0 || d_model <= 0 || n_layers <= 0 || !n_active_pad || !ksplit || bn < 32 || bn > 256 || bn % 32 != 0 ||
+      num_sms < 2 || !items || !n_items || !offsets)
+    return MLPMOE_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if (n_active_pad[l] <= 0 || n_active_pad[l] % 128 != 0 || ksplit[l] < 1 || ksplit[l] > 4) return MLPMOE_ERR_INVALID_ARG;
+  std::vector<int32_t> t, o;
+  std::vector<int> ks(ksplit, ksplit + n_layers);
+  tc_stack_schedule(n_tokens, d_model, n_active_pad, ks.data(), n_layers, bn, num_sms, &t, &o);
+  *n_items = static_cast<int64_t>(t.size() / 2);
+  if (static_cast<int64_t>(t.size() / 2) > item_capacity) return MLPMOE_ERR_INVALID_ARG;
+  std::memcpy(items, t.data(), sizeof(int32_t) * t.size());
+  std::memcpy(offsets, o.data(), sizeof(int32_t) * o.size());
   return MLPMOE_OK;
 }
 

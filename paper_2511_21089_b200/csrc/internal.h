@@ -127,6 +127,42 @@ int64_t tc_layer_schedule(int64_t n, int64_t d, int64_t Ipad, int bn, int ksplit
                           std::vector<int32_t>* offsets);
 cudaError_t launch_tc_layer(const TcLayerArgs& a, int num_sms, cudaStream_t st);
 
+// -------------------------------------------------------------- tc_stack.cu --
+// Whole pre-norm stack (n > 128) in one persistent CTA-pair kernel.  One record per layer in
+// device memory; work items are (code, layer) pairs, code = type << 30 | column << 16 | token block.
+constexpr int kItemGateUp = 0, kItemDown = 1, kItemNorm = 2;
+constexpr int kStackNormParts = 16;    // norm items per 256-token block
+struct alignas(64) TcStackLayer {
+  CUtensorMap tm_wgu;    // Wgu [2 Ipad x d]  bf16, box 64 x 128
+  CUtensorMap tm_h_st;   // H   [n x Ipad]    bf16, box 64 x 32
+  CUtensorMap tm_h_ld;   // H   [n x Ipad]    bf16, box 64 x 128
+  CUtensorMap tm_wdt;    // WdT [d x Ipad]    bf16, box 64 x bn/2
+  const float* scale;    // [Ipad]
+  int32_t n1;            // gate|up tiles per token block (Ipad / 128)
+  int32_t kb2;           // K-steps of the down GEMM (Ipad / 64)
+  int32_t ksplit;        // K slices per down tile
+  int32_t pad_[11];
+};
+struct TcStackArgs {
+  const TcStackLayer* layers;    // device, n_layers records
+  int n_layers;
+  CUtensorMap tm_x;      // Xn [n x d] bf16, box 64 x 128
+  CUtensorMap tm_y;      // x  [n x d] fp32, box 32 x 32
+  float* x;
+  void* xnorm;
+  int64_t n, d;
+  int bn;
+  float eps;
+  const int32_t* items;          // device: (code, layer) pairs, 8-byte aligned
+  const int32_t* list_offsets;   // device: [num_sms / 2 + 1], in items
+  uint32_t* counters;            // device: [3 x n_layers x ceil(n / 256)], zero at launch
+  uint32_t* status;
+};
+cudaError_t tc_stack_init();
+void tc_stack_schedule(int64_t n, int64_t d, const int64_t* Ipad, const int* ksplit, int n_layers, int bn, int num_sms,
+                       std::vector<int32_t>* items, std::vector<int32_t>* offsets);
+cudaError_t launch_tc_stack(const TcStackArgs& a, int num_sms, cudaStream_t st);
+
 // ---------------------------------------------------------------- decode.cu --
 struct DecodeArgs {
   CUtensorMap tm_w;     // Wgu [2*Ipad x d]  box 64 x 64

@@ -181,3 +181,58 @@ def test_tile_schedule_is_complete_and_cannot_deadlock(lib, n, d, Ipad, bn, ks):
     loads = [sum((Ipad // 64) * max(2 * bn, (16384 + bn * 64) // 50) // ks if t[0] else ((d + 63) // 64) * 655 for t in l) for l in lists]
     if m_pairs * (n1 + n2) >= 4 * 74:
         assert max(loads) <= 1.35 * (sum(loads) / len(loads))
+
+
+@pytest.mark.parametrize("n,d,Ipads,kss,bn", [(4096, 896, [3712, 3712, 4864], [3, 3, 2], 224), (300, 128, [256, 128], [1, 1], 128),
+                                              (2048, 4096, [14336, 11520], [1, 1], 256), (257, 896, [3712], [4], 224)])
+def test_stack_schedule_is_complete_and_cannot_deadlock(lib, n, d, Ipads, kss, bn):
+    """Every item of every layer exactly once; and whatever the items' real durations turn out to be,
+    running the sequences (per pair one of GEMM items and, independently, one of norm parts) under
+    the kernel's three waiting rules finishes: a norm part waits for all down items of its token
+    block in the previous layer, a gate|up tile for all norm parts of its block, a down item for
+    all gate|up tiles of its block."""
+    gemm, norm = lib.mlpmoe_host_stack_schedule(n, d, Ipads, kss, bn, 148)
+    assert all(t[0] != 2 for lst in gemm for t in lst) and all(t[0] == 2 for lst in norm for t in lst)
+    lists = gemm + norm
+    m_pairs, L = (n + 255) // 256, len(Ipads)
+    n2 = (d + bn - 1) // bn
+    want = set()
+    for l in range(L):
+        for m in range(m_pairs):
+            want |= {(2, part, m, l) for part in range(16)}
+            want |= {(0, nb, m, l) for nb in range(Ipads[l] // 128)}
+            want |= {(1, nb, m, l) for nb in range(n2 * kss[l])}
+    flat = [t for lst in lists for t in lst]
+    assert len(flat) == len(set(flat)) and set(flat) == want
+    need = {}                      # (kind it waits on, block, layer) -> arrivals needed
+    for l in range(L):
+        for m in range(m_pairs):
+            need[(2, m, l)] = 16
+            need[(0, m, l)] = Ipads[l] // 128
+            need[(1, m, l)] = n2 * kss[l]
+
+    def blocked(t, have):
+        typ, _, m, l = t
+        if typ == 2:
+            return l > 0 and have.get((1, m, l - 1), 0) < need[(1, m, l - 1)]
+        if typ == 0:
+            return have.get((2, m, l), 0) < need[(2, m, l)]
+        return have.get((0, m, l), 0) < need[(0, m, l)]
+
+    rng = np.random.default_rng(n)
+    for trial in range(2):
+        # the pair to advance is drawn at random among the runnable ones: any interleaving must finish
+        pos = [0] * len(lists)
+        have = {}
+        remaining = len(flat)
+        while remaining:
+            runnable = [c for c in range(len(lists)) if pos[c] < len(lists[c]) and not blocked(lists[c][pos[c]], have)]
+            assert runnable, "every pair is blocked: the schedule can deadlock"
+            for c in rng.permutation(runnable)[: max(1, len(runnable) // 2)]:
+                t = lists[c][pos[c]]
+                have[(t[0], t[2], t[3])] = have.get((t[0], t[2], t[3]), 0) + 1
+                pos[c] += 1
+                remaining -= 1
+    counts = [len(lst) for lst in gemm]
+    if len(flat) >= 8 * 74:
+        assert max(counts) <= 1.5 * (sum(counts) / len(counts)) + 4
