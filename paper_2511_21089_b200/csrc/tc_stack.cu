@@ -362,13 +362,12 @@ cudaError_t tc_stack_init() {
   return cudaFuncSetAttribute(tc_stack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
 }
 
-// Work sequences of every CTA pair for the whole stack.  One global order: layer after layer; in a
-// layer the norm parts of all token blocks, then the gate|up tiles token block after token block
-// (or in groups, see below), then the down items block after block.  GEMM items go, in that
-// order, to the pair with the least estimated work so far, so the deal keeps balancing across layer
-// boundaries; norm parts go round-robin to the pairs' norm warps.  Every sequence (a pair's GEMM
-// items; a pair's norm parts) is the global order restricted to its items and every item comes
-// after the items it waits for, so with all pairs resident the waits cannot form a cycle.
+// Work sequences of every CTA pair for the whole stack.  The GEMM items have one global order (a
+// stream over layers and token blocks, see below) and go, in that order, to the pair with the
+// least estimated work so far, so the deal keeps balancing across layer boundaries; norm parts go
+// round-robin, in (layer, block, part) order, to the pairs' norm warps.  Every sequence (a pair's
+// GEMM items; a pair's norm parts) is the global order restricted to its items and every item
+// comes after the items it waits for, so with all pairs resident the waits cannot form a cycle.
 // items: GEMM items of pair 0, 1, ... then norm items of pair 0, 1, ..., as (code, layer);
 // offsets: [pairs + 1] for the GEMM sequences followed by [pairs + 1] for the norm sequences.
 void tc_stack_schedule(int64_t n, int64_t d, const int64_t* Ipad, const int* ksplit, int n_layers, int bn, int num_sms,
@@ -396,27 +395,45 @@ void tc_stack_schedule(int64_t n, int64_t d, const int64_t* Ipad, const int* ksp
     next = (c + 1) % pairs;
   };
   int norm_next = 0;
-  for (int l = 0; l < n_layers; ++l) {
-    const int n1 = static_cast<int>(Ipad[l] / 128);
-    const int64_t cost_g = kb1 * kstep_cycles(256) + 1500;
-    const int64_t cost_d = (Ipad[l] / BK) * kstep_cycles(bn) / ksplit[l] + 1500 + 24 * bn;
+  for (int l = 0; l < n_layers; ++l)
     for (int m = 0; m < m_pairs; ++m)
       for (int part = 0; part < NORM_PARTS; ++part) {
         norm_lists[norm_next].push_back(encode_item(kItemNorm, part, m));
         norm_lists[norm_next].push_back(l);
         norm_next = (norm_next + 1) % pairs;
       }
-    // Weights that fit in L2 can be re-read at will: one token block after the other, so that blocks
-    // complete (and their down items become ready) one by one.  Larger weights are streamed from HBM
-    // once per group of 8 token blocks, the tiles of a group walking the weight tiles together.
-    const int group = 3 * d * Ipad[l] * 2 <= (int64_t(48) << 20) ? 1 : 8;
-    for (int g0 = 0; g0 < m_pairs; g0 += group) {
-      const int g1 = g0 + group < m_pairs ? g0 + group : m_pairs;
+  // The GEMM items as one stream over (layer, group of token blocks): slot s holds the gate|up tiles
+  // of its group and the down items of the group `lag` slots earlier, also across layer boundaries.
+  // A group is one token block when the layers' weights fit in L2 (they can be re-read at will) and
+  // 8 token blocks otherwise (the weights are streamed from HBM once per group, the tiles of a group
+  // walking the weight tiles together).  lag < groups per layer, so a block's down items still come
+  // before its gate|up tiles of the next layer.  The further back in the order the items that an
+  // item waits for, the less a pair that runs a little ahead of the others has to wait: 7/16 of the
+  // groups leaves the down items about as far behind their block's tiles as the next layer's tiles
+  // are behind the block's down items plus the time its norm takes.
+  bool fits_l2 = true;
+  for (int l = 0; l < n_layers; ++l) fits_l2 = fits_l2 && 3 * d * Ipad[l] * 2 <= (int64_t(48) << 20);
+  const int group = fits_l2 ? 1 : 8;
+  const int n_groups = (m_pairs + group - 1) / group;
+  int lag = (7 * n_groups + 8) / 16;
+  if (lag > n_groups - 1) lag = n_groups - 1;
+  const int slots = n_layers * n_groups;
+  for (int sl = 0; sl < slots + lag; ++sl) {
+    if (sl < slots) {
+      const int l = sl / n_groups, g = sl % n_groups;
+      const int n1 = static_cast<int>(Ipad[l] / 128);
+      const int64_t cost_g = kb1 * kstep_cycles(256) + 1500;
+      const int g0 = g * group, g1 = g0 + group < m_pairs ? g0 + group : m_pairs;
       for (int nb = 0; nb < n1; ++nb)
         for (int m = g0; m < g1; ++m) give(encode_item(kItemGateUp, nb, m), l, cost_g);
     }
-    for (int m = 0; m < m_pairs; ++m)
-      for (int nb = 0; nb < n2 * ksplit[l]; ++nb) give(encode_item(kItemDown, nb, m), l, cost_d);
+    if (sl >= lag) {
+      const int l = (sl - lag) / n_groups, g = (sl - lag) % n_groups;
+      const int64_t cost_d = (Ipad[l] / BK) * kstep_cycles(bn) / ksplit[l] + 1500 + 24 * bn;
+      const int g0 = g * group, g1 = g0 + group < m_pairs ? g0 + group : m_pairs;
+      for (int m = g0; m < g1; ++m)
+        for (int nb = 0; nb < n2 * ksplit[l]; ++nb) give(encode_item(kItemDown, nb, m), l, cost_d);
+    }
   }
   items->clear();
   offsets->clear();
