@@ -391,7 +391,8 @@ def run_ours(args):
             gu_ms = kms[0] / kcnt[0]
             dn_ms = kms[1] / max(kcnt[1], 1)
             fused = n > 128            # one kernel runs both GEMMs of a layer call
-            whole_stack = fused and w["stack"]     # ... and, for a stack, every layer and its RMSNorm
+            # ... and, for a stack of short layers, every layer and its RMSNorm (one launch per step)
+            whole_stack = fused and w["stack"] and int(kcnt[0]) == timed_steps
             if n > 64:
                 if whole_stack:
                     flops = float(np.sum(flops_gu)) + float(np.sum(flops_dn))

@@ -1,6 +1,7 @@
 // C-ABI entry points and the host side of the library: argument checks, the weight packer's
 // control flow, the branch scheduler (Section 3.3 -> K-list), Fade set-up (Section 3.2) and the
 // dispatch of mlpmoe_forward onto the prefill / decode / fp32 kernels.
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -751,9 +752,13 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
     return MLPMOE_OK;
   }
   if (layers[0]->dtype == MLPMOE_BF16 && n > 128 && n_layers <= kMaxStackLayers) {
-    bool same_ws = true;
-    for (int l = 1; l < n_layers; ++l) same_ws = same_ws && layers[l]->ws == layers[0]->ws;
-    if (same_ws) return prefill_stack(layers, n_layers, x, n, eps, st);
+    // The one-launch stack kernel pays where layers are short (weights that stay in L2: its gain is
+    // what a layer boundary costs); long layers run faster one launch per layer, on the cost-aware
+    // tile schedule of the single-layer kernel (measured on 4096 x 14336 layers).
+    bool use_stack = true;
+    for (int l = 0; l < n_layers; ++l)
+      use_stack = use_stack && layers[l]->ws == layers[0]->ws && 3 * layers[l]->d * layers[l]->Ipad * 2 <= kWeightsFitL2Bytes;
+    if (use_stack) return prefill_stack(layers, n_layers, x, n, eps, st);
   }
   for (int l = 0; l < n_layers; ++l) {
     mlpmoe_layer_s* h = layers[l];

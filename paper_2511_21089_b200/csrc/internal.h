@@ -36,6 +36,9 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 }
 
 constexpr int kGroup = 128;      // neurons per interleaved gate|up group in the packed operand
+// A layer's packed weights (3 * d_model * surviving neurons * 2 bytes) count as L2-resident below this size:
+// the prefill schedules may then re-read them at will instead of streaming them once per group of token blocks.
+constexpr int64_t kWeightsFitL2Bytes = int64_t(48) << 20;
 constexpr int kDecodeMaxTokens = 64;
 
 // Device status word values (written by kernels whose bounded waits run out).

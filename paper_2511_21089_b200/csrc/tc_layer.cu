@@ -355,7 +355,7 @@ int64_t tc_layer_schedule(int64_t n, int64_t d, int64_t Ipad, int bn, int ksplit
   // streamed from HBM once per group: take enough token blocks to keep every pair busy on one pass
   // over the weight tiles, and at least 8.
   int group = (pairs + n1 - 1) / n1 + 1;
-  const bool weights_fit_l2 = 3 * d * Ipad * 2 <= (int64_t(48) << 20);
+  const bool weights_fit_l2 = 3 * d * Ipad * 2 <= kWeightsFitL2Bytes;
   if (weights_fit_l2) group = 1;        // one token block after the other: blocks complete one by one, early
   else if (group < 8) group = 8;
   if (group > m_pairs) group = m_pairs;

@@ -412,7 +412,7 @@ void tc_stack_schedule(int64_t n, int64_t d, const int64_t* Ipad, const int* ksp
   // groups leaves the down items about as far behind their block's tiles as the next layer's tiles
   // are behind the block's down items plus the time its norm takes.
   bool fits_l2 = true;
-  for (int l = 0; l < n_layers; ++l) fits_l2 = fits_l2 && 3 * d * Ipad[l] * 2 <= (int64_t(48) << 20);
+  for (int l = 0; l < n_layers; ++l) fits_l2 = fits_l2 && 3 * d * Ipad[l] * 2 <= kWeightsFitL2Bytes;
   const int group = fits_l2 ? 1 : 8;
   const int n_groups = (m_pairs + group - 1) / group;
   int lag = (7 * n_groups + 8) / 16;
