@@ -87,12 +87,12 @@ def layer_inputs(layer: int, w):
     return bits, d_b, alpha, keep
 
 
-# DRAM traffic of one fused layer-kernel launch from the ncu capture summarised in
-# profiles/tc_layer_kernel_qwen_c2_2layers.md (dram__bytes_read.sum + dram__bytes_write.sum), valid
-# only while the kernel's sources are the ones that were profiled.
-GATEUP_TRAFFIC_BYTES = 42.16e6 + 4.08e6
+# DRAM traffic of one launch of the persistent prefill-stack kernel on the default workload, from the
+# ncu capture summarised in profiles/tc_stack_kernel_qwen_c2_24layers.md (dram__bytes_read.sum +
+# dram__bytes_write.sum), valid only while the kernel's sources are the ones that were profiled.
+GATEUP_TRAFFIC_BYTES = 889.68e6 + 969.74e6
 GATEUP_SOURCES = ("tc_stack.cu", "tc_common.cuh", "ptx.cuh")
-GATEUP_SOURCES_SHA = "058b6e7cb57620d0"
+GATEUP_SOURCES_SHA = "58173d7b1c1fb4c8"
 
 
 def gateup_traffic():
@@ -407,19 +407,25 @@ def run_ours(args):
                                    "achieved": achieved, "peak": pk["tflops_sustained"], "unit": "TFLOP/s",
                                    "frac": achieved / pk["tflops_sustained"], "traffic": gateup_traffic() if default else None,
                                    "peak_source": pk["source"] + " (sustained bf16 matmul)", "avg_launch_us": gu_ms * 1e3}
+            elif not w["stack"]:
+                # decode, one layer call: two kernels, each streams its part of the weights once
+                achieved = float(np.mean(wbytes_gu)) / (gu_ms * 1e-3) / 1e9
+                out["roofline"] = {"bound": "hbm", "kernel": "decode gate|up kernel (TMA weight ring + tcgen05)",
+                                   "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
+                                   "traffic": None, "peak_source": pk["source"] + " (copy bandwidth)", "avg_launch_us": gu_ms * 1e3}
             else:
                 # decode: one persistent kernel runs the whole stack and streams every layer's weights once
                 achieved = (sum(wbytes_gu) + sum(wbytes_dn)) / (gu_ms * 1e-3) / 1e9
                 out["roofline"] = {"bound": "hbm", "kernel": "persistent decode-stack kernel (TMA weight ring + tcgen05, all layers)",
                                    "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
                                    "traffic": None, "peak_source": pk["source"] + " (copy bandwidth)", "avg_launch_us": gu_ms * 1e3}
-            if n <= 64:
+            if n <= 64 and w["stack"]:
                 out["kernels"] = {"decode_stack": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_timed),
                                                    "weight_gbs": achieved}}
             elif whole_stack:
                 out["kernels"] = {"prefill_stack": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_timed),
                                                     "tflops": achieved}}
-            elif fused:
+            elif fused and n > 64:
                 out["kernels"] = {
                     "layer_fused": {"avg_us": gu_ms * 1e3, "launches": int(kcnt[0]), "share": float(kms[0] / ms_timed),
                                     "tflops": achieved},
