@@ -410,7 +410,9 @@ bool stack_kernel_ok() {
   static int state = -1;
   if (state < 0) {
     int per_sm = 0;
-    state = (decode_stack_init(&per_sm) == cudaSuccess && per_sm >= 1) ? 1 : 0;
+    int per_sm_fused = 0;
+    state = (decode_stack_init(&per_sm) == cudaSuccess && per_sm >= 1 && decode_fused_init(&per_sm_fused) == cudaSuccess &&
+             per_sm_fused >= 1) ? 1 : 0;
   }
   return state == 1;
 }
@@ -744,8 +746,14 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
     if (!make_tmap(&tm_x, h0->ws->xnorm, h0->d, n, h0->d, npad)) return MLPMOE_ERR_CUDA;
     CK(cudaMemsetAsync(h0->stack_counter, 0, sizeof(uint32_t) * 3 * n_layers, st));
     const long e0 = rec_event(h0, st);
-    CK(launch_decode_stack(h0->stack_dev, n_layers, tm_x, x, h0->ws->xnorm, n, h0->d, npad, eps, h0->stack_counter, h0->status,
-                           h0->num_sms, st));
+    if (n <= kDecodeFusedMaxTokens) {
+      // few tokens: both GEMMs of a layer on the CTA that owns the neurons (no H round trip, one dependency less per layer)
+      CK(launch_decode_fused(h0->stack_dev, n_layers, tm_x, x, h0->ws->xnorm, n, h0->d, eps, h0->stack_counter, h0->status,
+                             h0->num_sms, st));
+    } else {
+      CK(launch_decode_stack(h0->stack_dev, n_layers, tm_x, x, h0->ws->xnorm, n, h0->d, npad, eps, h0->stack_counter, h0->status,
+                             h0->num_sms, st));
+    }
     const long e1 = rec_event(h0, st);
     add_span(h0, SPAN_GATEUP, e0, e1);
     h0->launches += 1;
