@@ -175,6 +175,8 @@ struct mlpmoe_layer_s {
   DecodeStackLayer* stack_dev = nullptr;                    // layer records of the persistent decode-stack kernel
   uint32_t* stack_counter = nullptr;                        // its grid-wide event counter
   std::vector<DecodeStackLayer> stack_host;                 // what stack_dev currently holds
+  void* dec_tiled = nullptr;                                // stage-tiled weight copy of the fused few-token decode kernel,
+  int64_t dec_tiled_version = -1;                           //   built at the first such call after a (re)schedule
   // persistent prefill-stack kernel (buffers live in the first layer's handle, sized at the first call
   // with a new stack / token count)
   TcStackLayer* pstack_dev = nullptr;
@@ -228,7 +230,7 @@ void free_layer(mlpmoe_layer_s* h) {
   cudaFree(h->Wgu); cudaFree(h->WdT);
   cudaFree(h->scale); cudaFree(h->src_row); cudaFree(h->row_nnz);
   cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->block_done); cudaFree(h->tile_sched); cudaFree(h->stack_dev); cudaFree(h->stack_counter); cudaFree(h->status);
-  cudaFree(h->pstack_dev); cudaFree(h->pstack_items); cudaFree(h->pstack_counters);
+  cudaFree(h->pstack_dev); cudaFree(h->pstack_items); cudaFree(h->pstack_counters); cudaFree(h->dec_tiled);
   ws_release(h->ws);
   delete h;
 }
@@ -726,6 +728,22 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
     // decode: the whole stack in one persistent kernel (weights keep streaming across layer boundaries)
     mlpmoe_layer_s* h0 = layers[0];
     const int npad = n <= 16 ? 16 : (n <= 32 ? 32 : 64);
+    // Few tokens: the fused kernel, which streams a stage-tiled copy of the packed weights.  The copy
+    // (as large as the packed weights) is made at the first such call after a create / fade / prune;
+    // without memory for it the call runs on the other kernel.
+    bool fused = n <= kDecodeFusedMaxTokens;
+    for (int l = 0; fused && l < n_layers; ++l) {
+      mlpmoe_layer_s* h = layers[l];
+      if (h->dec_tiled != nullptr && h->dec_tiled_version == h->version) continue;
+      if (h->dec_tiled == nullptr && cudaMalloc(&h->dec_tiled, decode_tiled_bytes(h->Ipad_max, h->d)) != cudaSuccess) {
+        cudaGetLastError();
+        h->dec_tiled = nullptr;
+        fused = false;
+        break;
+      }
+      CK(launch_retile_decode(h->Wgu, h->WdT, h->dec_tiled, h->Ipad, h->d, st));
+      h->dec_tiled_version = h->version;
+    }
     std::vector<DecodeStackLayer> recs(static_cast<size_t>(n_layers));
     std::memset(recs.data(), 0, sizeof(DecodeStackLayer) * recs.size());
     for (int l = 0; l < n_layers; ++l) {
@@ -735,6 +753,7 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
       if (!make_tmap(&recs[l].tm_hd, h->ws->H, h->Ipad, n, h->Ipad, npad)) return MLPMOE_ERR_CUDA;
       recs[l].scale = h->scale;
       recs[l].Hd = static_cast<__nv_bfloat16*>(h->ws->H);
+      recs[l].tiled = fused ? static_cast<const uint8_t*>(h->dec_tiled) : nullptr;
       recs[l].Ipad = static_cast<int32_t>(h->Ipad);
     }
     if (h0->stack_host.size() != recs.size() ||
@@ -746,8 +765,8 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
     if (!make_tmap(&tm_x, h0->ws->xnorm, h0->d, n, h0->d, npad)) return MLPMOE_ERR_CUDA;
     CK(cudaMemsetAsync(h0->stack_counter, 0, sizeof(uint32_t) * 3 * n_layers, st));
     const long e0 = rec_event(h0, st);
-    if (n <= kDecodeFusedMaxTokens) {
-      // few tokens: both GEMMs of a layer on the CTA that owns the neurons (no H round trip, one dependency less per layer)
+    if (fused) {
+      // both GEMMs of a layer on the CTA that owns the neurons (no H round trip, one dependency less per layer)
       CK(launch_decode_fused(h0->stack_dev, n_layers, tm_x, x, h0->ws->xnorm, n, h0->d, eps, h0->stack_counter, h0->status,
                              h0->num_sms, st));
     } else {

@@ -69,6 +69,14 @@ struct FadeSeg {
 size_t fade_work_bytes(int nseg);
 cudaError_t launch_fade(const FadeSeg* segs_host, int nseg, void* work, int elem_size, cudaStream_t st);
 
+// Stage-tiled copy of the packed bf16 operands for the fused few-token decode kernel: per tile of 128
+// compacted neurons one contiguous run of 32 KB chunks, each the 128-byte-swizzled shared-memory image
+// of one stage (256 rows x 64 K): first ceil(d / 64) chunks of Wgu rows [256 t, 256 t + 256) (K-step
+// after K-step), then per block of 256 output columns two chunks of WdT[block rows, the tile's
+// neurons 0..63 | 64..127].  Rows / columns past d are zero.
+size_t decode_tiled_bytes(int64_t n_active_pad, int64_t d);
+cudaError_t launch_retile_decode(const void* Wgu, const void* WdT, void* tiled, int64_t n_active_pad, int64_t d, cudaStream_t st);
+
 // r = x / sqrt(mean(x^2) + eps), out bf16 (elem_size 2) or fp32 (4).
 cudaError_t launch_rmsnorm(const float* x, void* r, int64_t n, int64_t d, float eps, int out_elem_size, cudaStream_t st);
 
@@ -196,9 +204,11 @@ struct alignas(64) DecodeStackLayer {
   CUtensorMap tm_hd;     // Hd  [n x Ipad]    box 64 x npad
   const float* scale;    // [Ipad]
   __nv_bfloat16* Hd;     // [n x Ipad]
+  const uint8_t* tiled;  // stage-tiled weight copy of the fused few-token kernel (decode_tiled_bytes), else null
   int32_t Ipad;
-  int32_t pad_[11];
+  int32_t pad_[9];
 };
+static_assert(sizeof(DecodeStackLayer) == 448, "record layout");
 cudaError_t decode_stack_init(int* max_ctas_per_sm);
 cudaError_t launch_decode_stack(const DecodeStackLayer* layers_dev, int n_layers, const CUtensorMap& tm_x, float* x, void* xnorm,
                                 int64_t n, int64_t d, int npad, float eps, uint32_t* event_counter, uint32_t* status,

@@ -60,6 +60,30 @@ __global__ void gather_down_t_kernel(const T* __restrict__ Wd_c, const int32_t* 
   }
 }
 
+// ------------------------------------------- stage-tiled copy for decode ---
+// One thread per 16-byte piece of the destination.  A chunk is 256 rows of 128 bytes; piece c of row r
+// goes to piece position c ^ (r % 8) of that row (the 128-byte swizzle of the shared-memory tiles).
+__global__ void retile_decode_kernel(const uint4* __restrict__ Wgu, const uint4* __restrict__ WdT, uint4* __restrict__ out,
+                                     int64_t Ipad, int64_t d, int kb1, int m_blocks, int64_t total) {
+  const int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (q >= total) return;
+  const int chunks_per_tile = kb1 + 2 * m_blocks;
+  const int c = static_cast<int>(q % 8), r = static_cast<int>((q / 8) % 256);
+  const int64_t chunk_id = q / 2048;
+  const int chunk = static_cast<int>(chunk_id % chunks_per_tile);
+  const int64_t tile = chunk_id / chunks_per_tile;
+  uint4 v = make_uint4(0, 0, 0, 0);
+  if (chunk < kb1) {
+    const int64_t col = static_cast<int64_t>(chunk) * 64 + c * 8;                 // K coordinate (elements)
+    if (col < d) v = Wgu[((tile * 256 + r) * d + col) / 8];
+  } else {
+    const int blk = (chunk - kb1) / 2, ks = (chunk - kb1) % 2;
+    const int64_t row = static_cast<int64_t>(blk) * 256 + r;                      // output column of the layer
+    if (row < d) v = WdT[(row * Ipad + tile * 128 + ks * 64 + c * 8) / 8];
+  }
+  out[chunk_id * 2048 + r * 8 + (c ^ (r & 7))] = v;
+}
+
 // ------------------------------------------------------------ row nnz -------
 template <typename T>
 __device__ __forceinline__ bool is_nonzero(T v);
@@ -296,6 +320,20 @@ cudaError_t launch_row_nnz(const void* Wg_c, const void* Wu_c, const void* Wd_c,
   else
     row_nnz_kernel<uint32_t><<<blocks, 256, 0, st>>>(static_cast<const uint32_t*>(Wg_c), static_cast<const uint32_t*>(Wu_c),
                                                      static_cast<const uint32_t*>(Wd_c), out, I, d);
+  return cudaGetLastError();
+}
+
+size_t decode_tiled_bytes(int64_t n_active_pad, int64_t d) {
+  const int64_t chunks_per_tile = (d + 63) / 64 + 2 * ((d + 255) / 256);
+  return static_cast<size_t>(n_active_pad / 128 * chunks_per_tile) * 32768;
+}
+
+cudaError_t launch_retile_decode(const void* Wgu, const void* WdT, void* tiled, int64_t n_active_pad, int64_t d, cudaStream_t st) {
+  const int64_t total = static_cast<int64_t>(decode_tiled_bytes(n_active_pad, d) / 16);
+  if (total == 0) return cudaSuccess;
+  retile_decode_kernel<<<cdiv(total, 256), 256, 0, st>>>(static_cast<const uint4*>(Wgu), static_cast<const uint4*>(WdT),
+                                                        static_cast<uint4*>(tiled), n_active_pad, d,
+                                                        static_cast<int>((d + 63) / 64), static_cast<int>((d + 255) / 256), total);
   return cudaGetLastError();
 }
 
