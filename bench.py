@@ -88,8 +88,8 @@ def layer_inputs(layer: int, w):
 
 
 # DRAM traffic of one launch of the persistent prefill-stack kernel on the default workload, from the
-# ncu capture summarised in profiles/tc_stack_kernel_qwen_c2_24layers.md (dram__bytes_read.sum +
-# dram__bytes_write.sum), valid only while the kernel's sources are the ones that were profiled.
+# committed ncu summary of that kernel (dram__bytes_read.sum + dram__bytes_write.sum), valid only
+# while the kernel's sources are the ones that were profiled.
 GATEUP_TRAFFIC_BYTES = 889.68e6 + 969.74e6
 GATEUP_SOURCES = ("tc_stack.cu", "tc_common.cuh", "ptx.cuh")
 GATEUP_SOURCES_SHA = "58173d7b1c1fb4c8"
