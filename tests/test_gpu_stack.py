@@ -111,3 +111,42 @@ def test_config2_full_size_sampled_rows(lib):
     finally:
         for h in handles[1:] + handles[:1]:
             lib.mlpmoe_destroy(h)
+
+
+@pytest.mark.parametrize("n", [4, 40, 300])
+def test_stack_follows_a_later_prune_and_fade(lib, n):
+    """The stack kernels cache per-stack set-up (work sequences, layer records, the decode kernel's
+    tiled weight copy): a prune or a Fade between two calls must show in the second call."""
+    d, I, d_b, L = 256, 512, [128, 128, 64, 192], 2
+    cases, handles = [], []
+    try:
+        for l in range(L):
+            c = Case((207, l), d, I, d_b, bf16=True, std=0.05)
+            h = c.create(lib, 512)
+            if handles:
+                lib.mlpmoe_share_workspace(h, handles[0])
+            cases.append(c)
+            handles.append(h)
+        x = synth.normal_f32((207, 9, n), (n, d), 1.0)
+        ones = [1.0] * len(d_b)
+
+        def run_and_check(layers):
+            xd = dev_f32(x)
+            lib.mlpmoe_stack_forward(handles, xd, n, 1e-6, stream_ptr())
+            torch.cuda.synchronize()
+            ref = oracle.stack_forward(x, layers, bf16_activations=True)
+            assert rel_err(xd.cpu().numpy(), ref) <= TOL_BF16
+
+        run_and_check([(*c.host, d_b, ones) for c in cases])
+        keep = [True, False, True, True]
+        for h in handles:
+            lib.mlpmoe_prune(h, keep, True, stream_ptr())
+        run_and_check([(*c.host, d_b, oracle.prune_alpha(ones, keep)) for c in cases])
+        for h in handles:
+            lib.mlpmoe_fade(h, None, stream_ptr())
+        faded = [oracle.fade(c.host[0], c.host[1], d_b) for c in cases]
+        run_and_check([(Fg, Fu, c.host[2], d_b, oracle.prune_alpha(ones, keep)) for c, (Fg, Fu) in zip(cases, faded)])
+        assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
+    finally:
+        for h in handles[1:] + handles[:1]:
+            lib.mlpmoe_destroy(h)
