@@ -728,22 +728,23 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
     // decode: the whole stack in one persistent kernel (weights keep streaming across layer boundaries)
     mlpmoe_layer_s* h0 = layers[0];
     const int npad = n <= 16 ? 16 : (n <= 32 ? 32 : 64);
-    // Few tokens: the fused kernel, which streams a stage-tiled copy of the packed weights.  The copy
-    // (as large as the packed weights) is made at the first such call after a create / fade / prune;
-    // without memory for it the call runs on the other kernel.
-    bool fused = n <= kDecodeFusedMaxTokens;
-    for (int l = 0; fused && l < n_layers; ++l) {
+    // Both stack kernels stream a stage-tiled copy of the packed weights (contiguous 32 KB stage images).
+    // The copy (as large as the packed weights) is made at the first decode-stack call after a create /
+    // fade / prune; without memory for it the call reads the packed operands through tensor maps.
+    bool tiled = true;
+    for (int l = 0; tiled && l < n_layers; ++l) {
       mlpmoe_layer_s* h = layers[l];
       if (h->dec_tiled != nullptr && h->dec_tiled_version == h->version) continue;
       if (h->dec_tiled == nullptr && cudaMalloc(&h->dec_tiled, decode_tiled_bytes(h->Ipad_max, h->d)) != cudaSuccess) {
         cudaGetLastError();
         h->dec_tiled = nullptr;
-        fused = false;
+        tiled = false;
         break;
       }
       CK(launch_retile_decode(h->Wgu, h->WdT, h->dec_tiled, h->Ipad, h->d, st));
       h->dec_tiled_version = h->version;
     }
+    const bool fused = tiled && n <= kDecodeFusedMaxTokens;
     std::vector<DecodeStackLayer> recs(static_cast<size_t>(n_layers));
     std::memset(recs.data(), 0, sizeof(DecodeStackLayer) * recs.size());
     for (int l = 0; l < n_layers; ++l) {
@@ -753,7 +754,7 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
       if (!make_tmap(&recs[l].tm_hd, h->ws->H, h->Ipad, n, h->Ipad, npad)) return MLPMOE_ERR_CUDA;
       recs[l].scale = h->scale;
       recs[l].Hd = static_cast<__nv_bfloat16*>(h->ws->H);
-      recs[l].tiled = fused ? static_cast<const uint8_t*>(h->dec_tiled) : nullptr;
+      recs[l].tiled = tiled ? static_cast<const uint8_t*>(h->dec_tiled) : nullptr;
       recs[l].Ipad = static_cast<int32_t>(h->Ipad);
     }
     if (h0->stack_host.size() != recs.size() ||
