@@ -13,7 +13,7 @@
 // (Ipad / 128 x n x d_model fp32 atomics per layer), is small next to the weight stream.
 //
 // The CTAs beyond the number of tiles (36 of 148 at the Llama-8B shape) own no neurons; at every
-// layer boundary they request the next layer's first stages into L2 while HBM would idle (+1 to 4 %).
+// layer boundary they request the next layer's first stages into L2 while HBM would idle (+2 to 3.5 %).
 //
 // Warp roles as in decode_stack.cu: warp 0 TMA producer (it keeps issuing weight tiles across
 // events and only holds back the token tile of a phase A stage until event N has passed), warp 1
@@ -50,7 +50,7 @@ constexpr uint32_t TMEM_COLS = 128;                   // G | U (32 columns), the
 constexpr uint32_t ACC_B0 = 2 * NPAD;                 // first column of the phase B buffers
 constexpr uint64_t WAIT_NS = 1000000000ull;
 constexpr uint32_t ARRIVALS_PER_CTA = 4;              // every epilogue warp arrives once per event
-constexpr int HELPER_STAGES = 16;                     // stages per tile that a CTA without tiles requests into L2 at a layer boundary
+constexpr int HELPER_STAGES = 32;                     // stages per tile that a CTA without tiles requests into L2 at a layer boundary
 constexpr int NORM_VEC = 8;                           // float4 per lane the RMSNorm phase keeps in registers
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
@@ -153,10 +153,12 @@ decode_fused_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
         return true;
       };
       bool ok = true;
-      // A CTA without a tile in layer l + 1 helps the others over the layer boundary: when the first
-      // CTAs have finished layer l (HBM starts to idle while x is completed and normalised), it asks
-      // for the stages of layer l + 1 that lie just beyond the owners' rings to be brought into L2,
-      // from where the owners then refill their rings faster than HBM would serve them.
+      // A CTA without a tile in any layer helps the others over the layer boundaries: when three
+      // quarters of the owners have finished layer l (HBM starts to idle while x is completed and
+      // normalised), it asks for the stages of layer l + 1 that lie just beyond the owners' rings to be
+      // brought into L2, from where the owners then refill their rings faster than HBM would serve
+      // them.  Only where the owners are many enough to be bound by HBM (at least 70 % of the CTAs):
+      // with fewer owners each is bound by what one SM can take in, and the requests measured slower.
       int max_tiles = 0;
       for (int l = 0; l < n_layers; ++l) max_tiles = layers[l].Ipad / 128 > max_tiles ? layers[l].Ipad / 128 : max_tiles;
       if (cta >= max_tiles) {                              // no tile in any layer: this producer has nothing else to do
@@ -165,9 +167,11 @@ decode_fused_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
         for (int l = 0; ok && l + 1 < n_layers; ++l) {
           const DecodeStackLayer* Ln = layers + l + 1;
           const int tiles_next = Ln->Ipad / 128, tiles_this = layers[l].Ipad / 128;
-          // the CTAs without a tile in layer l arrive at its event B at once; one more arrival: the first owner is done
+          // (the CTAs without a tile in layer l arrive at its event B at once)
+          if (10 * tiles_next < 7 * ctas) continue;
           const uint32_t idle_arrivals = static_cast<uint32_t>(ctas - tiles_this) * ARRIVALS_PER_CTA;
-          if (!event_wait(event_counter + 2 * l + 1, idle_arrivals + ARRIVALS_PER_CTA, abort_flag)) { ok = false; break; }
+          const uint32_t owners_done = static_cast<uint32_t>(tiles_this) * 3u / 4u + 1u;
+          if (!event_wait(event_counter + 2 * l + 1, idle_arrivals + owners_done * ARRIVALS_PER_CTA, abort_flag)) { ok = false; break; }
           for (int tile = me; tile < tiles_next; tile += helpers)
             for (int s = STAGES; s < STAGES + HELPER_STAGES && s < kb1; ++s)
               bulk_prefetch_l2(Ln->tiled + (static_cast<int64_t>(tile) * cpt + s) * W_BYTES, W_BYTES);
