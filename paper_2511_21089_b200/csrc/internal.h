@@ -216,7 +216,7 @@ cudaError_t launch_decode_stack(const DecodeStackLayer* layers_dev, int n_layers
 
 // ----------------------------------------------------------- decode_fused.cu --
 // Decode stack for at most kDecodeFusedMaxTokens tokens: both GEMMs of a layer on the CTA that owns the neurons.
-constexpr int kDecodeFusedMaxTokens = 12;   // above, the partial sums per tile (fp32 atomics) cost more than the dependency saved (measured crossover 12..16)
+constexpr int kDecodeFusedMaxTokens = 13;   // above, the partial sums per tile (fp32 atomics) cost more than the dependency saved (measured: even at 14)
 cudaError_t decode_fused_init(int* max_ctas_per_sm);
 cudaError_t launch_decode_fused(const DecodeStackLayer* layers_dev, int n_layers, const CUtensorMap& tm_x, float* x, void* xnorm,
                                 int64_t n, int64_t d, float eps, uint32_t* event_counter, uint32_t* status, int num_sms,

@@ -52,8 +52,15 @@ def test_small_stack(lib, bf16, n):
         # host-buffer entry point
         yh = torch.empty((n, d), dtype=torch.float32)
         lib.mlpmoe_stack_forward_host(handles, torch.from_numpy(x), yh, n, 1e-6, stream_ptr())
-        # same numbers up to the order in which K slices are added into the fp32 stream
-        np.testing.assert_allclose(yh.numpy(), xd.cpu().numpy(), rtol=1e-5, atol=1e-5)
+        # Same numbers up to the order in which K slices are added into the fp32 stream.  In bf16 a
+        # last-bit difference of x can also flip the rounding of one normalised input of the next
+        # layer, which moves that token's row by a bf16 step of one product: far inside the parity
+        # tolerance, far outside fp32 round-off.
+        assert rel_err(yh.numpy(), ref) <= (TOL_BF16 if bf16 else TOL_FP32)
+        if bf16:
+            assert rel_err(yh.numpy(), xd.cpu().numpy().astype(np.float64)) <= TOL_BF16 / 4
+        else:
+            np.testing.assert_allclose(yh.numpy(), xd.cpu().numpy(), rtol=1e-5, atol=1e-5)
         assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
     finally:
         for h in handles[1:] + handles[:1]:
