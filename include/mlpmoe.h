@@ -160,6 +160,18 @@ mlpmoe_status_t mlpmoe_rmsnorm(const float* x, void* r, int64_t n_tokens, int64_
  * Run n_layers layers (all with the same d_model and dtype) over the fp32 residual
  * stream x [n_tokens x d_model], in place: for each layer, RMSNorm into a
  * library-owned buffer of the layer dtype, then x = x + MLPMoE_l(that).
+ *
+ * bf16 stacks whose layers share one workspace (mlpmoe_share_workspace) run in one
+ * persistent kernel: up to 64 tokens always, above 128 tokens when every layer's
+ * packed weights are small enough to stay in L2; other stacks run layer by layer.
+ * The first such call for a stack, a token count or a schedule (after create, fade
+ * or prune) does set-up work that later calls reuse: it builds the work sequences
+ * on the host, may allocate device memory for them (and, for up to 64 tokens, for a
+ * stage-tiled copy of each layer's packed weights, as large as the packed weights),
+ * and may synchronise `stream`; if that memory cannot be had, MLPMOE_ERR_ALLOC (above
+ * 128 tokens) or a slower kernel without the copy (up to 64 tokens).  Later calls
+ * only enqueue.  Work items add into x in arrival order, so the last bits of the
+ * result can differ from run to run.  x: device, 16-byte aligned.
  */
 mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_layers, float* x,
                                      int64_t n_tokens, float eps, void* stream);
