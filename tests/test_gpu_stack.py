@@ -29,7 +29,7 @@ def test_rmsnorm_kernel(lib):
 
 
 @pytest.mark.parametrize("bf16", [True, False])
-@pytest.mark.parametrize("n", [1, 5, 12, 13, 24, 300])
+@pytest.mark.parametrize("n", [1, 5, 12, 13, 14, 24, 64, 100, 129, 300, 512])
 def test_small_stack(lib, bf16, n):
     d, I, d_b, L = 256, 384, [128, 64, 192], 3
     cases, handles, layers = [], [], []
