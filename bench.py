@@ -441,6 +441,10 @@ def run_ours(args):
             }
         else:
             out["roofline"] = None
+        if out.get("roofline"):
+            # context only: the same figure against the nominal peaks (2.25 PFLOP/s dense bf16, 8 TB/s HBM3e)
+            nominal = 2250.0 if out["roofline"]["bound"] == "tensor" else 8000.0
+            out["roofline"]["frac_of_nominal"] = out["roofline"]["achieved"] / nominal
         if world == 1 and not args.no_cpu_baseline and w["name"] == "qwen_stack":
             rows = 512
             tps, dt = time_oracle(w, rows, 3, 1)
