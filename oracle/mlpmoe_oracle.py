@@ -116,20 +116,24 @@ def _as_fraction(s) -> Fraction:
 def fade_position(s, m: int) -> Tuple[int, Fraction]:
     """Position of the s-quantile among m sorted values (the usual linear
     definition): p = s (m - 1), split into the lower order statistic index
-    lo = floor(p) and the interpolation fraction p - lo.  Exact arithmetic."""
+    lo = floor(p) and the fraction p - lo.  Exact arithmetic."""
     p = _as_fraction(s) * (m - 1)
     lo = p.numerator // p.denominator
     return int(lo), p - lo
 
 
 def fade_mask(w: np.ndarray, s) -> np.ndarray:
-    """Keep-mask of one projection of one branch (Section 3.2 and the
-    'Differential Sparsity Logic' fragment of Section 4), step by step:
-        w_abs     = |w| as float32
-        threshold = s-quantile of all entries of w_abs (linear interpolation
-                    between the two neighbouring order statistics)
-        keep      = w_abs > threshold        (strict)
-    The threshold is evaluated in float64 from the float32 order statistics.
+    """Keep-mask of one projection of one branch under Fractal Fade (Section 3.2:
+    magnitude pruning of the slice at sparsity ratio s), stated by rank: with the
+    m magnitudes |w| (as float32) sorted ascending into a[0..m-1] and
+    lo = floor(s (m - 1)) in exact rational arithmetic, an entry is kept iff
+    |w| > a[lo].  Entries that tie with a[lo] go as well.
+
+    This is the set that the s-quantile threshold of Section 4 (linear
+    interpolation between a[lo] and a[lo+1], strict '>') selects: that threshold
+    t satisfies a[lo] <= t < a[lo+1] when the two differ and t = a[lo] otherwise,
+    so {|w| > t} = {|w| > a[lo]}; tests/test_oracle_fade_prune.py checks the
+    equivalence with the threshold evaluated in exact rationals.
     s == 0 means "leave untouched" (the paper's branch 0)."""
     s = _as_fraction(s)
     if not (0 <= s < 1):
@@ -139,15 +143,8 @@ def fade_mask(w: np.ndarray, s) -> np.ndarray:
         return np.ones(w.shape, dtype=bool)
     w_abs = np.abs(w.astype(np.float32))
     a = np.sort(w_abs, axis=None)
-    m = a.size
-    lo, frac = fade_position(s, m)
-    a_lo = float(a[lo])
-    if frac == 0:
-        threshold = a_lo
-    else:
-        a_hi = float(a[lo + 1])
-        threshold = a_lo + float(frac) * (a_hi - a_lo)
-    return w_abs.astype(np.float64) > threshold
+    lo, _ = fade_position(s, a.size)
+    return w_abs > a[lo]
 
 
 def fade(W_gate, W_up, d_b: Sequence[int], s: Optional[Sequence] = None):

@@ -116,6 +116,28 @@ def test_matches_the_papers_fragment_with_torch_quantile(s):
         assert np.array_equal(oracle.fade_mask(w, s), expect)
 
 
+def test_rank_form_equals_interpolated_threshold_in_exact_arithmetic():
+    """The rank form of fade_mask against the quantile threshold of Section 4 evaluated without
+    rounding: t = a[lo] + frac (a[lo+1] - a[lo]) in rationals, keep = |w| > t.  Includes ratios
+    whose double sits a hair below a rational (frac within 1e-16 of 1), where a float64
+    interpolation would round t up to a[lo+1] and drop one entry too many."""
+    rng = np.random.default_rng(11)
+    w = rng.standard_normal((9, 11)).astype(np.float32)
+    w[2, 3] = w[4, 5]                                            # a tie
+    m = w.size
+    a = np.sort(np.abs(w), axis=None)
+    ratios = [Fraction(1, 7), Fraction(9, 32), 0.3, 0.7, float(np.nextafter(20 / (m - 1), 0.0)), float(np.nextafter(0.5, 0.0))]
+    for s in ratios:
+        lo, frac = oracle.fade_position(s, m)
+        assert lo == (Fraction(s) * (m - 1)).__floor__()
+        a_lo, a_hi = Fraction(float(a[lo])), Fraction(float(a[min(lo + 1, m - 1)]))
+        t = a_lo + frac * (a_hi - a_lo)
+        expect = np.array([Fraction(float(v)) > t for v in np.abs(w).ravel()]).reshape(w.shape)
+        assert np.array_equal(oracle.fade_mask(w, s), expect), s
+    lo, frac = oracle.fade_position(float(np.nextafter(20 / (m - 1), 0.0)), m)
+    assert lo == 19 and 1 - frac < Fraction(1, 10 ** 12)         # the case a float64 interpolation gets wrong
+
+
 def test_ties_and_idempotence():
     w = np.array([[1, -1, 1, 2, 2, -3, 3, 4, 5, 6]], dtype=np.float32)
     keep = oracle.fade_mask(w, Fraction(1, 3))           # lo = 3 -> a[lo] = 2: both 2s go too
@@ -253,3 +275,26 @@ def test_rmsnorm_and_stack():
     np.testing.assert_allclose(inputs[1], x1, rtol=1e-13)
     # rows are independent: a subset of rows gives the same rows
     np.testing.assert_allclose(oracle.stack_forward(x[[1, 4]], layers), oracle.stack_forward(x, layers)[[1, 4]], rtol=1e-12)
+
+
+def test_stack_with_bf16_activations_hand_computed():
+    """Two layers of the pre-norm stack with the normalised input rounded to bfloat16, against values
+    derived by hand in tests/golden/tiny_stack_bf16.txt (the rounding of 1/sqrt(2) and of the second
+    layer's normalised input are where a missing or misplaced rounding shows)."""
+    g = {}
+    with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "tiny_stack_bf16.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                k, v = line.split()
+                g[k] = float(v)
+    c = math.log(3.0) * 128.0 / 181.0                        # bf16(sqrt 2) = 181/128, so the first gate pre-activation is ln 3
+    layer = (np.array([[c], [c]]), np.array([[1.0], [0.0]]), np.array([[1.0, 2.0]]), [1], [1.0])
+    x = np.array([[1.0, 0.0]])
+    y1, inputs = oracle.stack_forward(x, [layer], bf16_activations=True, eps=0.0, return_layer_inputs=True)
+    assert np.array_equal(inputs[0], x)
+    np.testing.assert_allclose(y1, [[g["layer1_x0"], g["layer1_x1"]]], rtol=1e-14)
+    y2 = oracle.stack_forward(x, [layer, layer], bf16_activations=True, eps=0.0)
+    np.testing.assert_allclose(y2, [[g["layer2_x0"], g["layer2_x1"]]], rtol=1e-14)
+    # without the rounding the layer's contribution moves in its 4th digit
+    y1_exact = oracle.stack_forward(x, [layer], bf16_activations=False, eps=0.0)
+    assert abs(y1_exact[0, 0] - g["layer1_x0"]) > 1e-4
