@@ -118,7 +118,9 @@ mlpmoe_status_t mlpmoe_prune_first_k(mlpmoe_handle_t h, int32_t K, void* stream)
 
 /* ------------------------------------------------------------------------- *
  * Forward (Section 3.1 layer equation).  Enqueues on `stream`, never
- * synchronises, allocates nothing.
+ * synchronises, allocates nothing.  (The first call above 128 tokens with a new
+ * token count builds that count's tile sequences on the host and uploads them
+ * with one asynchronous copy into memory sized at create.)
  * ------------------------------------------------------------------------- */
 
 /*
@@ -157,6 +159,19 @@ mlpmoe_status_t mlpmoe_rmsnorm(const float* x, void* r, int64_t n_tokens, int64_
                                mlpmoe_dtype_t out_dtype, void* stream);
 
 /*
+ * Set-up of mlpmoe_stack_forward for this stack (these handles, in this order) and this token
+ * count, so that the forward call itself only enqueues: chooses the kernel family, builds the work
+ * sequences on the host, allocates the device memory that holds them (and, for up to 64 tokens, a
+ * stage-tiled copy of each layer's packed weights, as large as the packed weights; if that memory
+ * cannot be had, a slower kernel without the copy), uploads them on `stream` and may synchronise
+ * `stream`.  The result is cached in the first layer's handle, one set-up at a time: preparing
+ * another token count or stack replaces it, and create / fade / prune on any layer invalidates it.
+ * Not in the paper: memory management only.  MLPMOE_ERR_ALLOC if the work sequences cannot be
+ * stored (above 128 tokens).
+ */
+mlpmoe_status_t mlpmoe_stack_prepare(const mlpmoe_handle_t* layers, int32_t n_layers, int64_t n_tokens, void* stream);
+
+/*
  * Run n_layers layers (all with the same d_model and dtype) over the fp32 residual
  * stream x [n_tokens x d_model], in place: for each layer, RMSNorm into a
  * library-owned buffer of the layer dtype, then x = x + MLPMoE_l(that).
@@ -164,13 +179,11 @@ mlpmoe_status_t mlpmoe_rmsnorm(const float* x, void* r, int64_t n_tokens, int64_
  * bf16 stacks whose layers share one workspace (mlpmoe_share_workspace) run in one
  * persistent kernel: up to 64 tokens always, above 128 tokens when every layer's
  * packed weights are small enough to stay in L2; other stacks run layer by layer.
- * The first such call for a stack, a token count or a schedule (after create, fade
- * or prune) does set-up work that later calls reuse: it builds the work sequences
- * on the host, may allocate device memory for them (and, for up to 64 tokens, for a
- * stage-tiled copy of each layer's packed weights, as large as the packed weights),
- * and may synchronise `stream`; if that memory cannot be had, MLPMOE_ERR_ALLOC (above
- * 128 tokens) or a slower kernel without the copy (up to 64 tokens).  Later calls
- * only enqueue.  Work items add into x in arrival order, so the last bits of the
+ * After mlpmoe_stack_prepare for the same stack and token count the call only
+ * enqueues: no allocation, no synchronisation.  Without it (or after a create / fade /
+ * prune, or with another token count) the call falls back to doing that set-up itself
+ * first, with everything mlpmoe_stack_prepare's comment says about allocation and
+ * synchronisation.  Work items add into x in arrival order, so the last bits of the
  * result can differ from run to run.  x: device, 16-byte aligned.
  */
 mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_layers, float* x,
@@ -207,9 +220,22 @@ mlpmoe_status_t mlpmoe_nnz(mlpmoe_handle_t h, int64_t* nnz_gate, int64_t* nnz_up
 mlpmoe_status_t mlpmoe_get_weights(mlpmoe_handle_t h, void* W_gate, void* W_up, void* W_down, void* stream);
 /*
  * Reads the handle's device status word (synchronises the device): MLPMOE_OK, or
- * MLPMOE_ERR_DEVICE_TIMEOUT if a bounded wait in a kernel expired since create.
+ * MLPMOE_ERR_DEVICE_TIMEOUT if a bounded wait in a kernel ran out since the last call (for a
+ * stack call the word of the first layer's handle is the one that is set).  The outputs of
+ * the call that timed out, and of every later call on the handle, are undefined until this
+ * function has reported the timeout: reporting it also re-arms the handle (clears the word and
+ * the dependency counters that a kernel which gave up may have left non-zero), after which
+ * the handle can be used again.
  */
 mlpmoe_status_t mlpmoe_get_status(mlpmoe_handle_t h);
+/*
+ * SM clock during the handle's last launch of a persistent kernel (the fused prefill kernel, the
+ * prefill-stack kernel, the decode-stack kernels; for a stack call ask the first layer's handle):
+ * one thread of the kernel reads the SM cycle counter and the nanosecond wall clock at entry and at
+ * exit; sm_mhz = cycles / nanoseconds * 1000, kernel_us = that thread's lifetime.  0 if no such kernel
+ * has run.  Synchronises the device.  For benchmarks (not in the paper).
+ */
+mlpmoe_status_t mlpmoe_get_kernel_clock(mlpmoe_handle_t h, double* sm_mhz, double* kernel_us);
 /* Kernels launched on behalf of this handle since create (forward calls only). */
 mlpmoe_status_t mlpmoe_get_launch_count(mlpmoe_handle_t h, int64_t* launches);
 const char* mlpmoe_status_string(mlpmoe_status_t s);
@@ -225,6 +251,30 @@ const char* mlpmoe_status_string(mlpmoe_status_t s);
  */
 mlpmoe_status_t mlpmoe_set_timing(mlpmoe_handle_t h, int32_t enable);
 mlpmoe_status_t mlpmoe_get_timing(mlpmoe_handle_t h, double* ms, int64_t* launches);
+
+/* ------------------------------------------------------------------------- *
+ * Hooks for tests (not in the paper)
+ * ------------------------------------------------------------------------- */
+
+/*
+ * Bounded-wait limits of the kernels launched for this handle (for a stack call: the first
+ * layer's handle).  limit_ns: how long a wait inside a kernel may last before the kernel gives
+ * up, sets the status word and returns (0 = the default of one second).  extra_arrivals is added
+ * to the number of arrivals that every wait of one CTA for the work of other CTAs expects; any
+ * value above 0 therefore makes those waits run out, which is how the tests reach the give-up
+ * path without a fault.  (0, 0) restores normal operation.
+ */
+mlpmoe_status_t mlpmoe_debug_set_wait(mlpmoe_handle_t h, uint64_t limit_ns, uint32_t extra_arrivals);
+
+/*
+ * The handle's (possibly shared) activation workspace, for guard-band checks and memory
+ * accounting: device addresses and sizes in bytes of H (n x n_active_pad of the layer dtype for
+ * an n-token call), of the normalised / staged input (n x d_model, layer dtype) and of the fp32
+ * staging buffer of the host-buffer calls (n x d_model), and the current padded neuron count.
+ * Any output may be NULL.  The memory stays owned by the library.
+ */
+mlpmoe_status_t mlpmoe_get_workspace(mlpmoe_handle_t h, void** H, int64_t* H_bytes, void** xnorm, int64_t* xnorm_bytes,
+                                     float** yres, int64_t* yres_bytes, int64_t* n_active_pad);
 
 /* ------------------------------------------------------------------------- *
  * Allocation-free variant (the paper has no counterpart: this is a deployment aid)
@@ -245,13 +295,14 @@ mlpmoe_status_t mlpmoe_get_timing(mlpmoe_handle_t h, double* ms, int64_t* launch
  * array of about 275 KB inside the library image, present on every device that loads the
  * library for the life of the process.  The call uses no cudaMalloc, cudaFree or other
  * allocating routine.
- *   slices, m, s   host arrays of length n_slices (slices holds device pointers).
+ *   slices, m, s   host arrays of length n_slices (slices holds device pointers, each aligned
+ *                  to the element size of `dtype`, else MLPMOE_ERR_INVALID_ARG).
  *   n_slices       at most MLPMOE_STATIC_FADE_MAX_SLICES, else MLPMOE_ERR_UNSUPPORTED.
  * The first call on each device looks up the array's device address (the device must be
- * current); make that first call outside any stream capture.  All calls share the one array:
- * each call re-initialises the part it uses, but two calls whose kernels overlap on the GPU
- * (different streams, or different host threads) race on it - serialise them.  Synchronises
- * `stream` before returning.
+ * current).  All calls share the one array: each call re-initialises the part it uses, but two
+ * calls whose kernels overlap on the GPU (different streams, or different host threads) race on
+ * it - serialise them.  Every call synchronises `stream` before it returns (its segment records
+ * are copied from host memory of the call), so it cannot be part of a stream capture.
  */
 mlpmoe_status_t mlpmoe_fade_buffers_static(void* const* slices, const int64_t* m, const double* s,
                                            int32_t n_slices, mlpmoe_dtype_t dtype, void* stream);

@@ -44,6 +44,10 @@ SIGNATURES = {
     "mlpmoe_forward_ex": (c_int32, [c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int32, c_void_p]),
     "mlpmoe_forward_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_int64, c_void_p]),
     "mlpmoe_rmsnorm": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_float, c_int32, c_void_p]),
+    "mlpmoe_stack_prepare": (c_int32, [POINTER(c_void_p), c_int32, c_int64, c_void_p]),
+    "mlpmoe_debug_set_wait": (c_int32, [c_void_p, ctypes.c_uint64, ctypes.c_uint32]),
+    "mlpmoe_get_workspace": (c_int32, [c_void_p, POINTER(c_void_p), POINTER(c_int64), POINTER(c_void_p), POINTER(c_int64),
+                                       POINTER(c_void_p), POINTER(c_int64), POINTER(c_int64)]),
     "mlpmoe_stack_forward": (c_int32, [POINTER(c_void_p), c_int32, c_void_p, c_int64, c_float, c_void_p]),
     "mlpmoe_stack_forward_host": (c_int32, [POINTER(c_void_p), c_int32, c_void_p, c_void_p, c_int64, c_float, c_void_p]),
     "mlpmoe_get_klist": (c_int32, [c_void_p, POINTER(c_int32), POINTER(c_int32), POINTER(c_int64), POINTER(c_int64),
@@ -53,6 +57,7 @@ SIGNATURES = {
     "mlpmoe_nnz": (c_int32, [c_void_p, POINTER(c_int64), POINTER(c_int64), POINTER(c_int64)]),
     "mlpmoe_get_weights": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "mlpmoe_get_status": (c_int32, [c_void_p]),
+    "mlpmoe_get_kernel_clock": (c_int32, [c_void_p, POINTER(c_double), POINTER(c_double)]),
     "mlpmoe_get_launch_count": (c_int32, [c_void_p, POINTER(c_int64)]),
     "mlpmoe_status_string": (c_char_p, [c_int32]),
     "mlpmoe_set_timing": (c_int32, [c_void_p, c_int32]),
@@ -170,6 +175,25 @@ def mlpmoe_stack_forward(layers: Sequence[int], x, n_tokens: int, eps: float = 1
     _check(lib.mlpmoe_stack_forward(arr, len(layers), _ptr(x), n_tokens, eps, _stream(stream)), "mlpmoe_stack_forward")
 
 
+def mlpmoe_stack_prepare(layers: Sequence[int], n_tokens: int, stream=None) -> None:
+    arr = (c_void_p * len(layers))(*layers)
+    _check(lib.mlpmoe_stack_prepare(arr, len(layers), n_tokens, _stream(stream)), "mlpmoe_stack_prepare")
+
+
+def mlpmoe_debug_set_wait(h: int, limit_ns: int = 0, extra_arrivals: int = 0) -> None:
+    _check(lib.mlpmoe_debug_set_wait(h, limit_ns, extra_arrivals), "mlpmoe_debug_set_wait")
+
+
+def mlpmoe_get_workspace(h: int) -> dict:
+    """Addresses and byte sizes of the handle's activation workspace, and the padded neuron count."""
+    H, xn, yr = c_void_p(), c_void_p(), c_void_p()
+    hb, xb, yb, ip = c_int64(), c_int64(), c_int64(), c_int64()
+    _check(lib.mlpmoe_get_workspace(h, ctypes.byref(H), ctypes.byref(hb), ctypes.byref(xn), ctypes.byref(xb), ctypes.byref(yr),
+                                    ctypes.byref(yb), ctypes.byref(ip)), "mlpmoe_get_workspace")
+    return dict(H=H.value, H_bytes=hb.value, xnorm=xn.value, xnorm_bytes=xb.value, yres=yr.value, yres_bytes=yb.value,
+                n_active_pad=ip.value)
+
+
 def mlpmoe_stack_forward_host(layers: Sequence[int], x_host, y_host, n_tokens: int, eps: float = 1e-6, stream=None) -> None:
     arr = (c_void_p * len(layers))(*layers)
     _check(lib.mlpmoe_stack_forward_host(arr, len(layers), _ptr(x_host), _ptr(y_host), n_tokens, eps, _stream(stream)),
@@ -211,6 +235,13 @@ def mlpmoe_get_weights(h: int, W_gate=None, W_up=None, W_down=None, stream=None)
 
 def mlpmoe_get_status(h: int) -> int:
     return lib.mlpmoe_get_status(h)
+
+
+def mlpmoe_get_kernel_clock(h: int):
+    """(SM MHz, kernel lifetime in microseconds) of the handle's last persistent-kernel launch."""
+    mhz, us = c_double(), c_double()
+    _check(lib.mlpmoe_get_kernel_clock(h, ctypes.byref(mhz), ctypes.byref(us)), "mlpmoe_get_kernel_clock")
+    return mhz.value, us.value
 
 
 def mlpmoe_get_launch_count(h: int) -> int:

@@ -2,6 +2,7 @@
 // control flow, the branch scheduler (Section 3.3 -> K-list), Fade set-up (Section 3.2) and the
 // dispatch of mlpmoe_forward onto the prefill / decode / fp32 kernels.
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -184,8 +185,15 @@ struct mlpmoe_layer_s {
   uint32_t* pstack_counters = nullptr;
   int64_t pstack_layer_cap = 0, pstack_item_cap = 0, pstack_counter_cap = 0, pstack_n_items = 0;
   int pstack_bn = 0;
-  std::vector<int64_t> pstack_key;                          // what the device buffers were built for
   int64_t version = 0;                                      // bumped by every reschedule
+  int64_t uid = 0;                                          // process-wide, never reused (a freed handle's address can be)
+  // what the last mlpmoe_stack_prepare / first mlpmoe_stack_forward set up for a stack that starts with this layer
+  std::vector<int64_t> plan_key;
+  int plan_kind = 0;                                        // PLAN_*
+  bool plan_fused = false;                                  // decode: the few-token kernel
+  int plan_npad = 0;
+  CUtensorMap plan_tm_x;                                    // normalised rows [n x d] as the kernels' token operand
+  WaitCfg wait;                                             // bounded-wait limits of this handle's launches (test hook)
   uint32_t* counters = nullptr;
   uint32_t* block_done = nullptr;                           // [2 x ceil(max_tokens / 256)] gate|up completion counters
   int64_t max_blocks = 0;
@@ -210,6 +218,7 @@ struct mlpmoe_layer_s {
 namespace {
 
 constexpr size_t kEventPool = 2048;
+constexpr size_t kStatusBytes = 64;        // status word, then (at byte 16) the clock probe of the last persistent-kernel launch
 constexpr int kMaxStackLayers = 256;       // layers one persistent decode-stack launch can take
 enum { SPAN_GATEUP = 0, SPAN_DOWN = 1, SPAN_RMSNORM = 2 };
 
@@ -277,6 +286,23 @@ mlpmoe_status_t reschedule(mlpmoe_layer_s* h, cudaStream_t st) {
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// The tile sequences of the fused prefill kernel for n tokens: chosen and uploaded (host work and one
+// asynchronous copy into a buffer sized at create) at the first call with this token count / output
+// mode since the last reschedule.
+mlpmoe_status_t ensure_tile_schedule(mlpmoe_layer_s* h, int64_t n, int bn, int out_mode, cudaStream_t st) {
+  if (h->sched_n == n && h->sched_Ipad == h->Ipad && h->sched_bn == bn && h->sched_out_mode == out_mode) return MLPMOE_OK;
+  const int ksplit = tc_layer_ksplit(n, h->d, h->Ipad, bn, out_mode, h->num_sms);
+  std::vector<int32_t> tiles, offs;
+  tc_layer_schedule(n, h->d, h->Ipad, bn, ksplit, h->num_sms, &tiles, &offs);
+  if (static_cast<int64_t>(tiles.size() + offs.size()) > h->sched_capacity) return MLPMOE_ERR_UNSUPPORTED;
+  h->sched_host = tiles;
+  h->sched_host.insert(h->sched_host.end(), offs.begin(), offs.end());
+  h->sched_tiles = static_cast<int>(tiles.size());
+  CK(cudaMemcpyAsync(h->tile_sched, h->sched_host.data(), sizeof(int32_t) * h->sched_host.size(), cudaMemcpyHostToDevice, st));
+  h->sched_n = n; h->sched_Ipad = h->Ipad; h->sched_bn = bn; h->sched_ksplit = ksplit; h->sched_out_mode = out_mode;
+  return MLPMOE_OK;
+}
 
 mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t n, const float* residual,
                              mlpmoe_dtype_t y_dtype, cudaStream_t st) {
@@ -354,25 +380,15 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
     a.Y = y;
     a.y_bf16 = y_dtype == MLPMOE_BF16;
     a.n = n; a.d = h->d; a.Ipad = h->Ipad;
-    if (h->sched_n != n || h->sched_Ipad != h->Ipad || h->sched_bn != a.bn || h->sched_out_mode != a.out_mode) {
-      // first call with this token count / output mode since the last reschedule: choose the K
-      // slicing, build the tile sequences (host work) and upload them
-      const int ksplit = tc_layer_ksplit(n, h->d, h->Ipad, a.bn, a.out_mode, h->num_sms);
-      std::vector<int32_t> tiles, offs;
-      tc_layer_schedule(n, h->d, h->Ipad, a.bn, ksplit, h->num_sms, &tiles, &offs);
-      if (static_cast<int64_t>(tiles.size() + offs.size()) > h->sched_capacity) return MLPMOE_ERR_UNSUPPORTED;
-      h->sched_host = tiles;
-      h->sched_host.insert(h->sched_host.end(), offs.begin(), offs.end());
-      h->sched_tiles = static_cast<int>(tiles.size());
-      CK(cudaMemcpyAsync(h->tile_sched, h->sched_host.data(), sizeof(int32_t) * h->sched_host.size(), cudaMemcpyHostToDevice, st));
-      h->sched_n = n; h->sched_Ipad = h->Ipad; h->sched_bn = a.bn; h->sched_ksplit = ksplit; h->sched_out_mode = a.out_mode;
-    }
+    mlpmoe_status_t src = ensure_tile_schedule(h, n, a.bn, a.out_mode, st);
+    if (src != MLPMOE_OK) return src;
     a.ksplit = h->sched_ksplit;
     a.tile_list = h->tile_sched;
     a.list_offsets = h->tile_sched + h->sched_tiles;
     a.done = h->block_done;
     a.passed = h->block_done + h->max_blocks;
     a.status = h->status;
+    a.wait = h->wait;
     const long e0 = rec_event(h, st);
     CK(launch_tc_layer(a, h->num_sms, st));
     const long e1 = rec_event(h, st);
@@ -429,82 +445,188 @@ mlpmoe_status_t check_stack(const mlpmoe_handle_t* layers, int32_t n_layers, int
   return MLPMOE_OK;
 }
 
-// Prefill of a stack whose layers share one workspace: the whole stack in one persistent CTA-pair
-// kernel.  The first call with a new stack, token count or schedule builds the work sequences on
-// the host and (re)sizes the device buffers that hold them; later calls only zero the counters
-// and launch.
-mlpmoe_status_t prefill_stack(const mlpmoe_handle_t* layers, int32_t n_layers, float* x, int64_t n, float eps, cudaStream_t st) {
+enum { PLAN_NONE = 0, PLAN_DECODE = 1, PLAN_PREFILL_STACK = 2, PLAN_PER_LAYER = 3 };
+
+// What a stack call's set-up depends on: the token count, the shared workspace, and every layer's identity
+// (a process-wide id, never reused) and schedule version.
+std::vector<int64_t> stack_key(const mlpmoe_handle_t* layers, int32_t n_layers, int64_t n) {
+  std::vector<int64_t> key;
+  key.reserve(4 + 2 * static_cast<size_t>(n_layers));
+  key.push_back(n);
+  key.push_back(n_layers);
+  key.push_back(reinterpret_cast<int64_t>(layers[0]->ws->H));
+  key.push_back(reinterpret_cast<int64_t>(layers[0]->ws->xnorm));
+  for (int l = 0; l < n_layers; ++l) {
+    key.push_back(layers[l]->uid);
+    key.push_back(layers[l]->version);
+  }
+  return key;
+}
+
+// Set-up of the persistent decode kernels for this stack and token count: the stage-tiled weight copies
+// (allocated at the first decode set-up of a layer, rebuilt after a reschedule), the layer records and
+// the token operand's tensor map.
+mlpmoe_status_t plan_decode(const mlpmoe_handle_t* layers, int32_t n_layers, int64_t n, cudaStream_t st) {
+  mlpmoe_layer_s* h0 = layers[0];
+  const int npad = n <= 16 ? 16 : (n <= 32 ? 32 : 64);
+  bool tiled = true;
+  for (int l = 0; tiled && l < n_layers; ++l) {
+    mlpmoe_layer_s* h = layers[l];
+    if (h->dec_tiled != nullptr && h->dec_tiled_version == h->version) continue;
+    if (h->dec_tiled == nullptr && cudaMalloc(&h->dec_tiled, decode_tiled_bytes(h->Ipad_max, h->d)) != cudaSuccess) {
+      cudaGetLastError();
+      h->dec_tiled = nullptr;
+      tiled = false;          // without memory for the copy the 14..64-token kernel reads the packed operands through tensor maps
+      break;
+    }
+    CK(launch_retile_decode(h->Wgu, h->WdT, h->dec_tiled, h->Ipad, h->d, st));
+    h->dec_tiled_version = h->version;
+  }
+  h0->stack_host.assign(static_cast<size_t>(n_layers), DecodeStackLayer());
+  std::memset(h0->stack_host.data(), 0, sizeof(DecodeStackLayer) * h0->stack_host.size());
+  for (int l = 0; l < n_layers; ++l) {
+    mlpmoe_layer_s* h = layers[l];
+    DecodeStackLayer& r = h0->stack_host[l];
+    r.tm_wgu = h->tm_wgu;
+    r.tm_wdt = h->tm_wdt256;
+    if (!make_tmap(&r.tm_hd, h->ws->H, h->Ipad, n, h->Ipad, npad)) return MLPMOE_ERR_CUDA;
+    r.scale = h->scale;
+    r.Hd = static_cast<__nv_bfloat16*>(h->ws->H);
+    r.tiled = tiled ? static_cast<const uint8_t*>(h->dec_tiled) : nullptr;
+    r.Ipad = static_cast<int32_t>(h->Ipad);
+  }
+  CK(cudaMemcpyAsync(h0->stack_dev, h0->stack_host.data(), sizeof(DecodeStackLayer) * h0->stack_host.size(), cudaMemcpyHostToDevice, st));
+  if (!make_tmap(&h0->plan_tm_x, h0->ws->xnorm, h0->d, n, h0->d, npad)) return MLPMOE_ERR_CUDA;
+  h0->plan_fused = tiled && n <= kDecodeFusedMaxTokens;
+  h0->plan_npad = npad;
+  return MLPMOE_OK;
+}
+
+// Set-up of the persistent prefill-stack kernel: the work sequences (host), the layer records, and the
+// device buffers that hold them (re-allocated when they are too small, which synchronises `st`).
+mlpmoe_status_t plan_prefill_stack(const mlpmoe_handle_t* layers, int32_t n_layers, int64_t n, cudaStream_t st) {
   mlpmoe_layer_s* h0 = layers[0];
   const int64_t d = h0->d;
   const int bn = tc_layer_down_bn(n, d, h0->num_sms);
   const int64_t m_pairs = (n + 255) / 256;
-  std::vector<int64_t> key;
-  key.reserve(4 + 2 * static_cast<size_t>(n_layers));
-  key.push_back(n);
-  key.push_back(bn);
-  key.push_back(reinterpret_cast<int64_t>(h0->ws->H));
-  key.push_back(reinterpret_cast<int64_t>(h0->ws->xnorm));
+  std::vector<TcStackLayer> recs(static_cast<size_t>(n_layers));
+  std::memset(recs.data(), 0, sizeof(TcStackLayer) * recs.size());
+  std::vector<int64_t> Ipad(n_layers);
+  std::vector<int> ksplit(n_layers);
   for (int l = 0; l < n_layers; ++l) {
-    key.push_back(reinterpret_cast<int64_t>(layers[l]));
-    key.push_back(layers[l]->version);
+    mlpmoe_layer_s* h = layers[l];
+    Ipad[l] = h->Ipad;
+    ksplit[l] = tc_layer_ksplit(n, d, h->Ipad, bn, TcLayerArgs::OUT_TMA_ADD, h0->num_sms);
+    recs[l].tm_wgu = h->tm_wgu_pair;
+    if (!make_tmap(&recs[l].tm_h_st, h->ws->H, h->Ipad, n, h->Ipad, 32)) return MLPMOE_ERR_CUDA;
+    if (!make_tmap(&recs[l].tm_h_ld, h->ws->H, h->Ipad, n, h->Ipad, 128)) return MLPMOE_ERR_CUDA;
+    if (!make_tmap(&recs[l].tm_wdt, h->WdT, h->Ipad, d, h->Ipad, bn / 2)) return MLPMOE_ERR_CUDA;
+    recs[l].scale = h->scale;
+    recs[l].n1 = static_cast<int32_t>(h->Ipad / 128);
+    recs[l].kb2 = static_cast<int32_t>(h->Ipad / 64);
+    recs[l].ksplit = ksplit[l];
   }
-  if (key != h0->pstack_key) {
-    std::vector<TcStackLayer> recs(static_cast<size_t>(n_layers));
-    std::memset(recs.data(), 0, sizeof(TcStackLayer) * recs.size());
-    std::vector<int64_t> Ipad(n_layers);
-    std::vector<int> ksplit(n_layers);
-    for (int l = 0; l < n_layers; ++l) {
-      mlpmoe_layer_s* h = layers[l];
-      Ipad[l] = h->Ipad;
-      ksplit[l] = tc_layer_ksplit(n, d, h->Ipad, bn, TcLayerArgs::OUT_TMA_ADD, h0->num_sms);
-      recs[l].tm_wgu = h->tm_wgu_pair;
-      if (!make_tmap(&recs[l].tm_h_st, h->ws->H, h->Ipad, n, h->Ipad, 32)) return MLPMOE_ERR_CUDA;
-      if (!make_tmap(&recs[l].tm_h_ld, h->ws->H, h->Ipad, n, h->Ipad, 128)) return MLPMOE_ERR_CUDA;
-      if (!make_tmap(&recs[l].tm_wdt, h->WdT, h->Ipad, d, h->Ipad, bn / 2)) return MLPMOE_ERR_CUDA;
-      recs[l].scale = h->scale;
-      recs[l].n1 = static_cast<int32_t>(h->Ipad / 128);
-      recs[l].kb2 = static_cast<int32_t>(h->Ipad / 64);
-      recs[l].ksplit = ksplit[l];
+  std::vector<int32_t> items, offs;
+  tc_stack_schedule(n, d, Ipad.data(), ksplit.data(), n_layers, bn, h0->num_sms, &items, &offs);
+  const int64_t need_items = static_cast<int64_t>(items.size() + offs.size());
+  const int64_t need_counters = 3 * static_cast<int64_t>(n_layers) * m_pairs;
+  if (need_items > h0->pstack_item_cap || need_counters > h0->pstack_counter_cap || n_layers > h0->pstack_layer_cap) {
+    CK(cudaStreamSynchronize(st));     // earlier launches may still read the old buffers
+    cudaFree(h0->pstack_items); cudaFree(h0->pstack_counters); cudaFree(h0->pstack_dev);
+    h0->pstack_items = nullptr; h0->pstack_counters = nullptr; h0->pstack_dev = nullptr;
+    h0->pstack_item_cap = h0->pstack_counter_cap = h0->pstack_layer_cap = 0;
+    if (cudaMalloc(reinterpret_cast<void**>(&h0->pstack_items), sizeof(int32_t) * need_items) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&h0->pstack_counters), sizeof(uint32_t) * need_counters) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&h0->pstack_dev), sizeof(TcStackLayer) * n_layers) != cudaSuccess) {
+      cudaGetLastError();
+      return MLPMOE_ERR_ALLOC;
     }
-    std::vector<int32_t> items, offs;
-    tc_stack_schedule(n, d, Ipad.data(), ksplit.data(), n_layers, bn, h0->num_sms, &items, &offs);
-    const int64_t need_items = static_cast<int64_t>(items.size() + offs.size());
-    const int64_t need_counters = 3 * static_cast<int64_t>(n_layers) * m_pairs;
-    if (need_items > h0->pstack_item_cap || need_counters > h0->pstack_counter_cap || n_layers > h0->pstack_layer_cap) {
-      CK(cudaStreamSynchronize(st));     // earlier launches may still read the old buffers
-      cudaFree(h0->pstack_items); cudaFree(h0->pstack_counters); cudaFree(h0->pstack_dev);
-      h0->pstack_items = nullptr; h0->pstack_counters = nullptr; h0->pstack_dev = nullptr;
-      h0->pstack_item_cap = h0->pstack_counter_cap = h0->pstack_layer_cap = 0;
-      h0->pstack_key.clear();
-      if (cudaMalloc(reinterpret_cast<void**>(&h0->pstack_items), sizeof(int32_t) * need_items) != cudaSuccess ||
-          cudaMalloc(reinterpret_cast<void**>(&h0->pstack_counters), sizeof(uint32_t) * need_counters) != cudaSuccess ||
-          cudaMalloc(reinterpret_cast<void**>(&h0->pstack_dev), sizeof(TcStackLayer) * n_layers) != cudaSuccess)
-        return MLPMOE_ERR_ALLOC;
-      h0->pstack_item_cap = need_items; h0->pstack_counter_cap = need_counters; h0->pstack_layer_cap = n_layers;
-    }
-    items.insert(items.end(), offs.begin(), offs.end());
-    h0->pstack_n_items = static_cast<int64_t>(items.size() - offs.size());
-    CK(cudaMemcpyAsync(h0->pstack_items, items.data(), sizeof(int32_t) * items.size(), cudaMemcpyHostToDevice, st));
-    CK(cudaMemcpyAsync(h0->pstack_dev, recs.data(), sizeof(TcStackLayer) * recs.size(), cudaMemcpyHostToDevice, st));
-    CK(cudaStreamSynchronize(st));       // the host vectors above go out of scope
-    h0->pstack_key = key;
-    h0->pstack_bn = bn;
+    h0->pstack_item_cap = need_items; h0->pstack_counter_cap = need_counters; h0->pstack_layer_cap = n_layers;
   }
+  items.insert(items.end(), offs.begin(), offs.end());
+  h0->pstack_n_items = static_cast<int64_t>(items.size() - offs.size());
+  CK(cudaMemcpyAsync(h0->pstack_items, items.data(), sizeof(int32_t) * items.size(), cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(h0->pstack_dev, recs.data(), sizeof(TcStackLayer) * recs.size(), cudaMemcpyHostToDevice, st));
+  CK(cudaStreamSynchronize(st));       // the host vectors above go out of scope
+  if (!make_tmap(&h0->plan_tm_x, h0->ws->xnorm, d, n, d, 128)) return MLPMOE_ERR_CUDA;
+  h0->pstack_bn = bn;
+  return MLPMOE_OK;
+}
+
+// Which kernel family runs this stack call, and its set-up.  Cached in the first layer's handle under
+// stack_key(); a call with another stack, token count, workspace or schedule version plans again.
+mlpmoe_status_t plan_stack(const mlpmoe_handle_t* layers, int32_t n_layers, int64_t n, cudaStream_t st) {
+  mlpmoe_layer_s* h0 = layers[0];
+  std::vector<int64_t> key = stack_key(layers, n_layers, n);
+  if (h0->plan_kind != PLAN_NONE && key == h0->plan_key) return MLPMOE_OK;
+  h0->plan_kind = PLAN_NONE;
+  h0->plan_key.clear();
+  int kind = PLAN_PER_LAYER;
+  if (h0->dtype == MLPMOE_BF16 && n <= kDecodeMaxTokens && n_layers <= kMaxStackLayers && h0->d <= 32768 && stack_kernel_ok()) {
+    // decode: the whole stack in one persistent kernel (weights keep streaming across layer boundaries)
+    kind = PLAN_DECODE;
+  } else if (h0->dtype == MLPMOE_BF16 && n > 128 && n_layers <= kMaxStackLayers) {
+    // The one-launch stack kernel pays where layers are short (weights that stay in L2: its gain is
+    // what a layer boundary costs); long layers run faster one launch per layer, on the cost-aware
+    // tile schedule of the single-layer kernel (measured on 4096 x 14336 layers).
+    bool use_stack = true;
+    for (int l = 0; l < n_layers; ++l)
+      use_stack = use_stack && layers[l]->ws == h0->ws && 3 * layers[l]->d * layers[l]->Ipad * 2 <= kWeightsFitL2Bytes;
+    if (use_stack) kind = PLAN_PREFILL_STACK;
+  }
+  mlpmoe_status_t rc = MLPMOE_OK;
+  if (kind == PLAN_DECODE) {
+    rc = plan_decode(layers, n_layers, n, st);
+  } else if (kind == PLAN_PREFILL_STACK) {
+    rc = plan_prefill_stack(layers, n_layers, n, st);
+  } else if (h0->dtype == MLPMOE_BF16 && n > 128) {
+    // one fused-kernel launch per layer: choose and upload every layer's tile sequences now
+    for (int l = 0; rc == MLPMOE_OK && l < n_layers; ++l)
+      rc = ensure_tile_schedule(layers[l], n, tc_layer_down_bn(n, layers[l]->d, layers[l]->num_sms), TcLayerArgs::OUT_TMA_ADD, st);
+  }
+  if (rc != MLPMOE_OK) return rc;
+  h0->plan_kind = kind;
+  h0->plan_key = std::move(key);
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t run_decode_stack(const mlpmoe_handle_t* layers, int32_t n_layers, float* x, int64_t n, float eps, cudaStream_t st) {
+  mlpmoe_layer_s* h0 = layers[0];
+  CK(cudaMemsetAsync(h0->stack_counter, 0, sizeof(uint32_t) * 3 * n_layers, st));
+  const long e0 = rec_event(h0, st);
+  if (h0->plan_fused) {
+    // both GEMMs of a layer on the CTA that owns the neurons (no H round trip, one dependency less per layer)
+    CK(launch_decode_fused(h0->stack_dev, n_layers, h0->plan_tm_x, x, h0->ws->xnorm, n, h0->d, eps, h0->stack_counter, h0->status,
+                           h0->num_sms, h0->wait, st));
+  } else {
+    CK(launch_decode_stack(h0->stack_dev, n_layers, h0->plan_tm_x, x, h0->ws->xnorm, n, h0->d, h0->plan_npad, eps, h0->stack_counter,
+                           h0->status, h0->num_sms, h0->wait, st));
+  }
+  const long e1 = rec_event(h0, st);
+  add_span(h0, SPAN_GATEUP, e0, e1);
+  h0->launches += 1;
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t run_prefill_stack(const mlpmoe_handle_t* layers, int32_t n_layers, float* x, int64_t n, float eps, cudaStream_t st) {
+  mlpmoe_layer_s* h0 = layers[0];
+  const int64_t m_pairs = (n + 255) / 256;
   TcStackArgs a;
   a.layers = h0->pstack_dev;
   a.n_layers = n_layers;
-  if (!make_tmap(&a.tm_x, h0->ws->xnorm, d, n, d, 128)) return MLPMOE_ERR_CUDA;
-  if (!make_tmap_t(&a.tm_y, x, d, n, d, 32, 4)) return MLPMOE_ERR_CUDA;
+  a.tm_x = h0->plan_tm_x;
+  if (!make_tmap_t(&a.tm_y, x, h0->d, n, h0->d, 32, 4)) return MLPMOE_ERR_CUDA;     // x is the caller's: encoded per call
   a.x = x;
   a.xnorm = h0->ws->xnorm;
   a.n = n;
-  a.d = d;
-  a.bn = bn;
+  a.d = h0->d;
+  a.bn = h0->pstack_bn;
   a.eps = eps;
   a.items = h0->pstack_items;
   a.list_offsets = h0->pstack_items + h0->pstack_n_items;
   a.counters = h0->pstack_counters;
   a.status = h0->status;
+  a.wait = h0->wait;
   pdl_overlap_enabled() = !h0->timing;
   CK(cudaMemsetAsync(h0->pstack_counters, 0, sizeof(uint32_t) * 3 * n_layers * m_pairs, st));
   const long e0 = rec_event(h0, st);
@@ -545,6 +667,8 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
 
   mlpmoe_layer_s* h = new (std::nothrow) mlpmoe_layer_s();
   if (!h) return MLPMOE_ERR_ALLOC;
+  static std::atomic<int64_t> next_uid{1};
+  h->uid = next_uid.fetch_add(1);
   h->device = dev;
   h->num_sms = prop.multiProcessorCount;
   h->d = d_model;
@@ -591,7 +715,7 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
        cudaMalloc(reinterpret_cast<void**>(&h->stack_counter), sizeof(uint32_t) * 3 * kMaxStackLayers) == cudaSuccess &&
        cudaMalloc(&h->block_done, sizeof(uint32_t) * 2 * h->max_blocks) == cudaSuccess &&
        cudaMalloc(&h->tile_sched, sizeof(int32_t) * h->sched_capacity) == cudaSuccess &&
-       cudaMalloc(&h->status, sizeof(uint32_t)) == cudaSuccess &&
+       cudaMalloc(&h->status, kStatusBytes) == cudaSuccess &&
        cudaMalloc(&h->ws->H, static_cast<size_t>(max_tokens) * h->Ipad_max * es) == cudaSuccess &&
        cudaMalloc(&h->ws->xnorm, static_cast<size_t>(max_tokens) * d_model * es) == cudaSuccess &&
        cudaMalloc(reinterpret_cast<void**>(&h->ws->yres), static_cast<size_t>(max_tokens) * d_model * sizeof(float)) == cudaSuccess;
@@ -604,7 +728,7 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
   auto fail = [&](mlpmoe_status_t s) { free_layer(h); return s; };
   if (cudaMemsetAsync(h->counters, 0, sizeof(uint32_t) * m_blocks * 4, st) != cudaSuccess ||
       cudaMemsetAsync(h->block_done, 0, sizeof(uint32_t) * 2 * h->max_blocks, st) != cudaSuccess ||
-      cudaMemsetAsync(h->status, 0, sizeof(uint32_t), st) != cudaSuccess)
+      cudaMemsetAsync(h->status, 0, kStatusBytes, st) != cudaSuccess)
     return fail(MLPMOE_ERR_CUDA);
   // canonical copies: one row of d contiguous weights per intermediate neuron, for all three matrices
   cudaError_t e;
@@ -716,6 +840,13 @@ mlpmoe_status_t mlpmoe_rmsnorm(const float* x, void* r, int64_t n_tokens, int64_
   return MLPMOE_OK;
 }
 
+mlpmoe_status_t mlpmoe_stack_prepare(const mlpmoe_handle_t* layers, int32_t n_layers, int64_t n, void* stream) {
+  mlpmoe_status_t rc = check_stack(layers, n_layers, n);
+  if (rc != MLPMOE_OK) return rc;
+  if (n == 0) return MLPMOE_OK;
+  return plan_stack(layers, n_layers, n, static_cast<cudaStream_t>(stream));
+}
+
 mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_layers, float* x, int64_t n, float eps,
                                      void* stream) {
   mlpmoe_status_t rc = check_stack(layers, n_layers, n);
@@ -723,71 +854,11 @@ mlpmoe_status_t mlpmoe_stack_forward(const mlpmoe_handle_t* layers, int32_t n_la
   if (n == 0) return MLPMOE_OK;
   if (!x || !aligned16(x)) return MLPMOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (layers[0]->dtype == MLPMOE_BF16 && n <= kDecodeMaxTokens && n_layers <= kMaxStackLayers && layers[0]->d <= 32768 &&
-      stack_kernel_ok()) {
-    // decode: the whole stack in one persistent kernel (weights keep streaming across layer boundaries)
-    mlpmoe_layer_s* h0 = layers[0];
-    const int npad = n <= 16 ? 16 : (n <= 32 ? 32 : 64);
-    // Both stack kernels stream a stage-tiled copy of the packed weights (contiguous 32 KB stage images).
-    // The copy (as large as the packed weights) is made at the first decode-stack call after a create /
-    // fade / prune; without memory for it the call reads the packed operands through tensor maps.
-    bool tiled = true;
-    for (int l = 0; tiled && l < n_layers; ++l) {
-      mlpmoe_layer_s* h = layers[l];
-      if (h->dec_tiled != nullptr && h->dec_tiled_version == h->version) continue;
-      if (h->dec_tiled == nullptr && cudaMalloc(&h->dec_tiled, decode_tiled_bytes(h->Ipad_max, h->d)) != cudaSuccess) {
-        cudaGetLastError();
-        h->dec_tiled = nullptr;
-        tiled = false;
-        break;
-      }
-      CK(launch_retile_decode(h->Wgu, h->WdT, h->dec_tiled, h->Ipad, h->d, st));
-      h->dec_tiled_version = h->version;
-    }
-    const bool fused = tiled && n <= kDecodeFusedMaxTokens;
-    std::vector<DecodeStackLayer> recs(static_cast<size_t>(n_layers));
-    std::memset(recs.data(), 0, sizeof(DecodeStackLayer) * recs.size());
-    for (int l = 0; l < n_layers; ++l) {
-      mlpmoe_layer_s* h = layers[l];
-      recs[l].tm_wgu = h->tm_wgu;
-      recs[l].tm_wdt = h->tm_wdt256;
-      if (!make_tmap(&recs[l].tm_hd, h->ws->H, h->Ipad, n, h->Ipad, npad)) return MLPMOE_ERR_CUDA;
-      recs[l].scale = h->scale;
-      recs[l].Hd = static_cast<__nv_bfloat16*>(h->ws->H);
-      recs[l].tiled = tiled ? static_cast<const uint8_t*>(h->dec_tiled) : nullptr;
-      recs[l].Ipad = static_cast<int32_t>(h->Ipad);
-    }
-    if (h0->stack_host.size() != recs.size() ||
-        std::memcmp(h0->stack_host.data(), recs.data(), sizeof(DecodeStackLayer) * recs.size()) != 0) {
-      h0->stack_host = recs;
-      CK(cudaMemcpyAsync(h0->stack_dev, h0->stack_host.data(), sizeof(DecodeStackLayer) * recs.size(), cudaMemcpyHostToDevice, st));
-    }
-    CUtensorMap tm_x;
-    if (!make_tmap(&tm_x, h0->ws->xnorm, h0->d, n, h0->d, npad)) return MLPMOE_ERR_CUDA;
-    CK(cudaMemsetAsync(h0->stack_counter, 0, sizeof(uint32_t) * 3 * n_layers, st));
-    const long e0 = rec_event(h0, st);
-    if (fused) {
-      // both GEMMs of a layer on the CTA that owns the neurons (no H round trip, one dependency less per layer)
-      CK(launch_decode_fused(h0->stack_dev, n_layers, tm_x, x, h0->ws->xnorm, n, h0->d, eps, h0->stack_counter, h0->status,
-                             h0->num_sms, st));
-    } else {
-      CK(launch_decode_stack(h0->stack_dev, n_layers, tm_x, x, h0->ws->xnorm, n, h0->d, npad, eps, h0->stack_counter, h0->status,
-                             h0->num_sms, st));
-    }
-    const long e1 = rec_event(h0, st);
-    add_span(h0, SPAN_GATEUP, e0, e1);
-    h0->launches += 1;
-    return MLPMOE_OK;
-  }
-  if (layers[0]->dtype == MLPMOE_BF16 && n > 128 && n_layers <= kMaxStackLayers) {
-    // The one-launch stack kernel pays where layers are short (weights that stay in L2: its gain is
-    // what a layer boundary costs); long layers run faster one launch per layer, on the cost-aware
-    // tile schedule of the single-layer kernel (measured on 4096 x 14336 layers).
-    bool use_stack = true;
-    for (int l = 0; l < n_layers; ++l)
-      use_stack = use_stack && layers[l]->ws == layers[0]->ws && 3 * layers[l]->d * layers[l]->Ipad * 2 <= kWeightsFitL2Bytes;
-    if (use_stack) return prefill_stack(layers, n_layers, x, n, eps, st);
-  }
+  // a no-op after mlpmoe_stack_prepare for this stack and token count; otherwise the set-up happens here
+  rc = plan_stack(layers, n_layers, n, st);
+  if (rc != MLPMOE_OK) return rc;
+  if (layers[0]->plan_kind == PLAN_DECODE) return run_decode_stack(layers, n_layers, x, n, eps, st);
+  if (layers[0]->plan_kind == PLAN_PREFILL_STACK) return run_prefill_stack(layers, n_layers, x, n, eps, st);
   for (int l = 0; l < n_layers; ++l) {
     mlpmoe_layer_s* h = layers[l];
     pdl_overlap_enabled() = !h->timing;
@@ -873,7 +944,45 @@ mlpmoe_status_t mlpmoe_get_status(mlpmoe_handle_t h) {
   uint32_t w = 0;
   CK(cudaDeviceSynchronize());
   CK(cudaMemcpy(&w, h->status, sizeof(w), cudaMemcpyDeviceToHost));
-  return w == kStatusOk ? MLPMOE_OK : MLPMOE_ERR_DEVICE_TIMEOUT;
+  if (w == kStatusOk) return MLPMOE_OK;
+  // A kernel gave up: the dependency counters that its work items leave at zero in a normal run may hold
+  // anything.  Re-arm the handle (the counters that are not zeroed before every launch, and the status word).
+  CK(cudaMemset(h->block_done, 0, sizeof(uint32_t) * 2 * h->max_blocks));
+  CK(cudaMemset(h->counters, 0, sizeof(uint32_t) * ((h->d + 127) / 128) * 4));
+  CK(cudaMemset(h->status, 0, sizeof(uint32_t)));
+  return MLPMOE_ERR_DEVICE_TIMEOUT;
+}
+
+mlpmoe_status_t mlpmoe_debug_set_wait(mlpmoe_handle_t h, uint64_t limit_ns, uint32_t extra_arrivals) {
+  if (!h) return MLPMOE_ERR_INVALID_ARG;
+  h->wait = WaitCfg();
+  if (limit_ns != 0) h->wait.limit_ns = limit_ns;
+  h->wait.extra_arrivals = extra_arrivals;
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_get_workspace(mlpmoe_handle_t h, void** H, int64_t* H_bytes, void** xnorm, int64_t* xnorm_bytes,
+                                     float** yres, int64_t* yres_bytes, int64_t* n_active_pad) {
+  if (!h) return MLPMOE_ERR_INVALID_ARG;
+  const Workspace* w = h->ws;
+  if (H) *H = w->H;
+  if (H_bytes) *H_bytes = w->max_tokens * w->Ipad_max * w->elem_size;
+  if (xnorm) *xnorm = w->xnorm;
+  if (xnorm_bytes) *xnorm_bytes = w->max_tokens * w->d * w->elem_size;
+  if (yres) *yres = w->yres;
+  if (yres_bytes) *yres_bytes = w->max_tokens * w->d * static_cast<int64_t>(sizeof(float));
+  if (n_active_pad) *n_active_pad = h->Ipad;
+  return MLPMOE_OK;
+}
+
+mlpmoe_status_t mlpmoe_get_kernel_clock(mlpmoe_handle_t h, double* sm_mhz, double* kernel_us) {
+  if (!h) return MLPMOE_ERR_INVALID_ARG;
+  uint64_t probe[2] = {0, 0};
+  CK(cudaDeviceSynchronize());
+  CK(cudaMemcpy(probe, reinterpret_cast<const char*>(h->status) + 16, sizeof(probe), cudaMemcpyDeviceToHost));
+  if (sm_mhz) *sm_mhz = probe[1] ? static_cast<double>(probe[0]) / static_cast<double>(probe[1]) * 1e3 : 0.0;
+  if (kernel_us) *kernel_us = static_cast<double>(probe[1]) * 1e-3;
+  return MLPMOE_OK;
 }
 
 mlpmoe_status_t mlpmoe_get_launch_count(mlpmoe_handle_t h, int64_t* launches) {

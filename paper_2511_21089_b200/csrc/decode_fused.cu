@@ -48,7 +48,6 @@ static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA m
 static_assert(HBUF_BYTES % 1024 == 0 && STAGE_BYTES % 1024 == 0, "swizzled tiles start on 1024-byte boundaries");
 constexpr uint32_t TMEM_COLS = 128;                   // G | U (32 columns), then 2 buffers x 2 halves x 16 for phase B
 constexpr uint32_t ACC_B0 = 2 * NPAD;                 // first column of the phase B buffers
-constexpr uint64_t WAIT_NS = 1000000000ull;
 constexpr uint32_t ARRIVALS_PER_CTA = 4;              // every epilogue warp arrives once per event
 constexpr int HELPER_STAGES = 32;                     // stages per tile that a CTA without tiles requests into L2 at a layer boundary
 constexpr int NORM_VEC = 8;                           // float4 per lane the RMSNorm phase keeps in registers
@@ -67,7 +66,8 @@ __device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, 
 __device__ __forceinline__ bool event_passed(const uint32_t* counter, uint32_t target) {
   return ld_acquire_u32(counter) >= target;
 }
-__device__ __forceinline__ bool event_wait(const uint32_t* counter, uint32_t target, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool event_wait(const uint32_t* counter, uint32_t target, volatile uint32_t* abort_flag,
+                                           uint64_t WAIT_NS) {
   if (event_passed(counter, target)) return true;
   const uint64_t t0 = globaltimer_ns();
   uint32_t polls = 0;
@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 decode_fused_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
                     const __grid_constant__ CUtensorMap tm_x,   // xnorm [n x d] bf16, box 64 x 16
                     float* x, __nv_bfloat16* xnorm, int64_t n, int64_t d, float eps, uint32_t* event_counter,
-                    uint32_t* status) {
+                    uint32_t* status, uint64_t WAIT_NS, uint32_t extra_arrivals) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem);
@@ -99,12 +99,13 @@ decode_fused_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
   uint64_t* tempty_b = tfull_b + 2;                     // [2] phase B buffer read (4 epilogue warps)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_b + 2);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  const ClockProbe probe = clock_probe_begin();
   volatile float* norm_part = reinterpret_cast<volatile float*>(tmem_slot + 4);   // one partial sum of squares per epilogue warp
   uint8_t* hbuf = smem + BAR_BYTES;
   uint8_t* ring = smem + RING_OFFSET;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int cta = blockIdx.x, ctas = gridDim.x;
-  const uint32_t per_event = static_cast<uint32_t>(ctas) * ARRIVALS_PER_CTA;
+  const uint32_t per_event = static_cast<uint32_t>(ctas) * ARRIVALS_PER_CTA + extra_arrivals;   // extra: 0 outside tests
   const int m_blocks = static_cast<int>((d + 255) / 256);     // phase B: blocks of 256 output columns
   const int kb1 = static_cast<int>((d + BK - 1) / BK);
 
@@ -142,7 +143,7 @@ decode_fused_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
           const int h = def_head;
           if (!gate_is_open(def_layer[h])) {
             if (!block) return true;
-            if (!event_wait(event_counter + 2 * def_layer[h], per_event, abort_flag)) return false;
+            if (!event_wait(event_counter + 2 * def_layer[h], per_event, abort_flag, WAIT_NS)) return false;
             block = false;
             continue;
           }
@@ -171,7 +172,7 @@ decode_fused_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
           if (10 * tiles_next < 7 * ctas) continue;
           const uint32_t idle_arrivals = static_cast<uint32_t>(ctas - tiles_this) * ARRIVALS_PER_CTA;
           const uint32_t owners_done = static_cast<uint32_t>(tiles_this) * 3u / 4u + 1u;
-          if (!event_wait(event_counter + 2 * l + 1, idle_arrivals + owners_done * ARRIVALS_PER_CTA, abort_flag)) { ok = false; break; }
+          if (!event_wait(event_counter + 2 * l + 1, idle_arrivals + owners_done * ARRIVALS_PER_CTA, abort_flag, WAIT_NS)) { ok = false; break; }
           for (int tile = me; tile < tiles_next; tile += helpers)
             for (int s = STAGES; s < STAGES + HELPER_STAGES && s < kb1; ++s)
               bulk_prefetch_l2(Ln->tiled + (static_cast<int64_t>(tile) * cpt + s) * W_BYTES, W_BYTES);
@@ -292,7 +293,7 @@ decode_fused_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
       const int Ipad = L->Ipad;
       // ---- phase N: x is final once every CTA has added the parts of its tiles of the previous layer
       if (ok && l > 0) {
-        bool w = event_wait(event_counter + 2 * l - 1, per_event, abort_flag);
+        bool w = event_wait(event_counter + 2 * l - 1, per_event, abort_flag, WAIT_NS);
         ok = __all_sync(0xFFFFFFFFu, w);
       }
       for (int t = cta; t < n; t += ctas) {
@@ -403,6 +404,7 @@ decode_fused_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
   __syncthreads();
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, TMEM_COLS); }
   if (threadIdx.x == 0 && *abort_flag) atomicExch(status, kStatusTimeout);
+  if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe_end(status, probe);
 }
 
 }  // namespace
@@ -417,11 +419,13 @@ cudaError_t decode_fused_init(int* max_ctas_per_sm) {
 // (the caller uses it up to kDecodeFusedMaxTokens).
 cudaError_t launch_decode_fused(const DecodeStackLayer* layers_dev, int n_layers, const CUtensorMap& tm_x, float* x, void* xnorm,
                                 int64_t n, int64_t d, float eps, uint32_t* event_counter, uint32_t* status, int num_sms,
-                                cudaStream_t st) {
+                                const WaitCfg& wait, cudaStream_t st) {
   if (n == 0 || n_layers == 0) return cudaSuccess;
   __nv_bfloat16* xn = static_cast<__nv_bfloat16*>(xnorm);
+  uint64_t wait_ns = wait.limit_ns;
+  uint32_t extra = wait.extra_arrivals;
   void* args[] = {const_cast<DecodeStackLayer**>(&layers_dev), &n_layers, const_cast<CUtensorMap*>(&tm_x), &x, &xn, &n, &d,
-                  &eps, &event_counter, &status};
+                  &eps, &event_counter, &status, &wait_ns, &extra};
   // cooperative launch: the grid-wide events need every CTA resident at once
   return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(decode_fused_kernel), dim3(num_sms), dim3(NUM_THREADS), args,
                                      SMEM_BYTES, st);

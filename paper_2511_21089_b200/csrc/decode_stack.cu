@@ -45,7 +45,6 @@ __host__ __device__ constexpr int stages_for(int npad) {
   return RING_BYTES / stage_bytes_for(npad) < MAX_STAGES ? RING_BYTES / stage_bytes_for(npad) : MAX_STAGES;
 }
 constexpr uint32_t TMEM_COLS = 4 * MAXN;              // 2 buffers x (G | U)
-constexpr uint64_t WAIT_NS = 1000000000ull;
 constexpr uint32_t ARRIVALS_PER_CTA = 4;              // every epilogue warp arrives once per event
 constexpr int NORM_VEC = 8;                           // float4 per lane the RMSNorm phase keeps in registers
 
@@ -65,7 +64,8 @@ __device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, 
 __device__ __forceinline__ bool event_passed(const uint32_t* counter, uint32_t target) {
   return ld_acquire_u32(counter) >= target;
 }
-__device__ __forceinline__ bool event_wait(const uint32_t* counter, uint32_t target, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool event_wait(const uint32_t* counter, uint32_t target, volatile uint32_t* abort_flag,
+                                           uint64_t WAIT_NS) {
   if (event_passed(counter, target)) return true;
   const uint64_t t0 = globaltimer_ns();
   uint32_t polls = 0;
@@ -179,7 +179,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
                     const __grid_constant__ CUtensorMap tm_x,   // xnorm [n x d] bf16, box 64 x npad
                     float* x, __nv_bfloat16* xnorm, int64_t n, int64_t d, int npad, float eps, uint32_t* event_counter,
-                    uint32_t* status) {
+                    uint32_t* status, uint64_t WAIT_NS, uint32_t extra_arrivals) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem);
@@ -188,10 +188,11 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
   uint64_t* tempty_bar = tfull_bar + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  const ClockProbe probe = clock_probe_begin();
   volatile float* norm_part = reinterpret_cast<volatile float*>(tmem_slot + 4);   // one partial sum of squares per epilogue warp
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int cta = blockIdx.x, ctas = gridDim.x;
-  const uint32_t per_event = static_cast<uint32_t>(ctas) * ARRIVALS_PER_CTA;
+  const uint32_t per_event = static_cast<uint32_t>(ctas) * ARRIVALS_PER_CTA + extra_arrivals;   // extra: 0 outside tests
   const int m_blocks = static_cast<int>((d + 255) / 256);     // phase B: blocks of 256 output columns
   const int kb1 = static_cast<int>((d + BK - 1) / BK);
 
@@ -235,7 +236,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
         if (ev != gate_ev) {
           // a new phase: the deferred tiles of the previous one go first (events pass in order)
           if (deferred > 0) {
-            if (!event_wait(event_counter + gate_ev, per_event, abort_flag)) { ok = false; break; }
+            if (!event_wait(event_counter + gate_ev, per_event, abort_flag, WAIT_NS)) { ok = false; break; }
             flush();
           }
           gate_ev = ev;
@@ -243,7 +244,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
           def_map = cur.ph == 0 ? &tm_x : &layers[cur.l].tm_hd;
         }
         if (!gate_open && (deferred == STAGES || event_passed(event_counter + gate_ev, per_event))) {
-          if (deferred == STAGES && !event_wait(event_counter + gate_ev, per_event, abort_flag)) { ok = false; break; }
+          if (deferred == STAGES && !event_wait(event_counter + gate_ev, per_event, abort_flag, WAIT_NS)) { ok = false; break; }
           flush();
         }
         if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, WAIT_NS)) { ok = false; break; }
@@ -260,7 +261,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         cur.advance();
       }
-      if (ok && deferred > 0 && event_wait(event_counter + gate_ev, per_event, abort_flag)) flush();
+      if (ok && deferred > 0 && event_wait(event_counter + gate_ev, per_event, abort_flag, WAIT_NS)) flush();
     }
   }
   else if (warp == 1) {
@@ -333,7 +334,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
       const int Ipad = L->Ipad;
       // ---- phase N: x is final once every K slice of the previous layer has been added
       if (ok && l > 0) {
-        bool w = event_wait(event_counter + 3 * l - 1, per_event, abort_flag);
+        bool w = event_wait(event_counter + 3 * l - 1, per_event, abort_flag, WAIT_NS);
         ok = __all_sync(0xFFFFFFFFu, w);
       }
       for (int t = cta; t < n; t += ctas) {
@@ -443,6 +444,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
   __syncthreads();
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, TMEM_COLS); }
   if (threadIdx.x == 0 && *abort_flag) atomicExch(status, kStatusTimeout);
+  if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe_end(status, probe);
 }
 
 }  // namespace
@@ -456,11 +458,13 @@ cudaError_t decode_stack_init(int* max_ctas_per_sm) {
 // layers_dev: n_layers records in device memory (64-byte aligned).  event_counter: 3 * n_layers zeros.
 cudaError_t launch_decode_stack(const DecodeStackLayer* layers_dev, int n_layers, const CUtensorMap& tm_x, float* x, void* xnorm,
                                 int64_t n, int64_t d, int npad, float eps, uint32_t* event_counter, uint32_t* status,
-                                int num_sms, cudaStream_t st) {
+                                int num_sms, const WaitCfg& wait, cudaStream_t st) {
   if (n == 0 || n_layers == 0) return cudaSuccess;
   __nv_bfloat16* xn = static_cast<__nv_bfloat16*>(xnorm);
+  uint64_t wait_ns = wait.limit_ns;
+  uint32_t extra = wait.extra_arrivals;
   void* args[] = {const_cast<DecodeStackLayer**>(&layers_dev), &n_layers, const_cast<CUtensorMap*>(&tm_x), &x, &xn, &n, &d, &npad,
-                  &eps, &event_counter, &status};
+                  &eps, &event_counter, &status, &wait_ns, &extra};
   // cooperative launch: the grid-wide events need every CTA resident at once
   return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(decode_stack_kernel), dim3(num_sms), dim3(NUM_THREADS), args,
                                      SMEM_BYTES, st);

@@ -41,6 +41,14 @@ constexpr int kGroup = 128;      // neurons per interleaved gate|up group in the
 constexpr int64_t kWeightsFitL2Bytes = int64_t(48) << 20;
 constexpr int kDecodeMaxTokens = 64;
 
+// Limits of the bounded waits of one launch.  Ordinary launches use the defaults; the test hook
+// mlpmoe_debug_set_wait shortens the limit and adds `extra_arrivals` to the target of every wait of
+// one CTA for work of other CTAs, so that such a wait runs out and the give-up path can be tested.
+struct WaitCfg {
+  uint64_t limit_ns = 1000000000ull;
+  uint32_t extra_arrivals = 0;
+};
+
 // Device status word values (written by kernels whose bounded waits run out).
 constexpr uint32_t kStatusOk = 0;
 constexpr uint32_t kStatusTimeout = 1;
@@ -130,6 +138,7 @@ struct TcLayerArgs {
   uint32_t* done;        // [ceil(n / 256)] zero between calls
   uint32_t* passed;      // [ceil(n / 256)] zero between calls
   uint32_t* status;
+  WaitCfg wait;
 };
 cudaError_t tc_layer_init();
 int tc_layer_down_bn(int64_t n, int64_t d, int num_sms);
@@ -168,6 +177,7 @@ struct TcStackArgs {
   const int32_t* list_offsets;   // device: [num_sms / 2 + 1], in items
   uint32_t* counters;            // device: [3 x n_layers x ceil(n / 256)], zero at launch
   uint32_t* status;
+  WaitCfg wait;
 };
 cudaError_t tc_stack_init();
 void tc_stack_schedule(int64_t n, int64_t d, const int64_t* Ipad, const int* ksplit, int n_layers, int bn, int num_sms,
@@ -212,7 +222,7 @@ static_assert(sizeof(DecodeStackLayer) == 448, "record layout");
 cudaError_t decode_stack_init(int* max_ctas_per_sm);
 cudaError_t launch_decode_stack(const DecodeStackLayer* layers_dev, int n_layers, const CUtensorMap& tm_x, float* x, void* xnorm,
                                 int64_t n, int64_t d, int npad, float eps, uint32_t* event_counter, uint32_t* status,
-                                int num_sms, cudaStream_t st);
+                                int num_sms, const WaitCfg& wait, cudaStream_t st);
 
 // ----------------------------------------------------------- decode_fused.cu --
 // Decode stack for at most kDecodeFusedMaxTokens tokens: both GEMMs of a layer on the CTA that owns the neurons.
@@ -220,6 +230,6 @@ constexpr int kDecodeFusedMaxTokens = 13;   // above, the partial sums per tile 
 cudaError_t decode_fused_init(int* max_ctas_per_sm);
 cudaError_t launch_decode_fused(const DecodeStackLayer* layers_dev, int n_layers, const CUtensorMap& tm_x, float* x, void* xnorm,
                                 int64_t n, int64_t d, float eps, uint32_t* event_counter, uint32_t* status, int num_sms,
-                                cudaStream_t st);
+                                const WaitCfg& wait, cudaStream_t st);
 
 }  // namespace mlpmoe

@@ -18,6 +18,24 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
   return t;
 }
 
+// SM cycle counter and wall clock of one thread at kernel entry; clock_probe_end stores the two
+// differences behind the status word (status[4..7] as two uint64: SM cycles, nanoseconds), from which the
+// host derives the SM clock the kernel really ran at.  Called by one thread of CTA 0 of a persistent kernel.
+struct ClockProbe {
+  uint64_t cycles, ns;
+};
+__device__ __forceinline__ ClockProbe clock_probe_begin() {
+  ClockProbe b;
+  b.cycles = static_cast<uint64_t>(clock64());
+  b.ns = globaltimer_ns();
+  return b;
+}
+__device__ __forceinline__ void clock_probe_end(uint32_t* status, const ClockProbe& b) {
+  uint64_t* out = reinterpret_cast<uint64_t*>(status + 4);
+  out[0] = static_cast<uint64_t>(clock64()) - b.cycles;
+  out[1] = globaltimer_ns() - b.ns;
+}
+
 // ------------------------------------------- programmatic dependent launch --
 // wait: blocks until every kernel this launch depends on has completed and its writes are
 // visible (a no-op for a launch without the programmatic-serialization attribute).

@@ -55,11 +55,14 @@ extern "C" mlpmoe_status_t mlpmoe_fade_buffers_static(void* const* slices, const
   if (dtype != MLPMOE_BF16 && dtype != MLPMOE_FP32) return MLPMOE_ERR_INVALID_ARG;
   if (n_slices > kMaxSlices) return MLPMOE_ERR_UNSUPPORTED;          // more slices than the fixed scratch holds
   if (fade_work_bytes(n_slices) > kScratchBytes) return MLPMOE_ERR_UNSUPPORTED;
+  const int elem_size = dtype == MLPMOE_BF16 ? 2 : 4;
   std::vector<FadeSeg> segs;
   segs.reserve(static_cast<size_t>(n_slices));
   for (int i = 0; i < n_slices; ++i) {
     if (!(s[i] >= 0.0 && s[i] < 1.0)) return MLPMOE_ERR_BAD_SCHEDULE;
     if (m[i] < 0 || (m[i] > 0 && !slices[i])) return MLPMOE_ERR_INVALID_ARG;
+    // the kernels read the slice as 2- or 4-byte words: an address off that grid would fault on the device
+    if (reinterpret_cast<uintptr_t>(slices[i]) % static_cast<uintptr_t>(elem_size) != 0) return MLPMOE_ERR_INVALID_ARG;
     if (s[i] == 0.0 || m[i] == 0) continue;                            // "leave untouched"
     int64_t lo = 0;
     if (mlpmoe_host_fade_position(s[i], m[i], &lo) != MLPMOE_OK) return MLPMOE_ERR_INVALID_ARG;
@@ -76,7 +79,7 @@ extern "C" mlpmoe_status_t mlpmoe_fade_buffers_static(void* const* slices, const
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // launch_fade re-initialises every record it uses (rank, prefix, histograms), so what an
   // earlier call left in the array does not matter.
-  if (launch_fade(segs.data(), static_cast<int>(segs.size()), scratch, dtype == MLPMOE_BF16 ? 2 : 4, st) != cudaSuccess)
+  if (launch_fade(segs.data(), static_cast<int>(segs.size()), scratch, elem_size, st) != cudaSuccess)
     return MLPMOE_ERR_CUDA;
   // the segment records were copied from this function's host memory
   if (cudaStreamSynchronize(st) != cudaSuccess) return MLPMOE_ERR_CUDA;

@@ -45,7 +45,6 @@ constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;
 static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 constexpr int ACC_STRIDE = 256;                      // TMEM columns per accumulator buffer
 constexpr int TMEM_COLS = 512;
-constexpr uint64_t WAIT_NS = 1000000000ull;
 constexpr uint32_t ARRIVALS_PER_GATEUP_TILE = 8;     // 4 epilogue warps in each of the two CTAs
 
 struct LayerParams {
@@ -64,6 +63,8 @@ struct LayerParams {
   uint32_t* done;         // [m_pairs] finished gate|up tile arrivals; zero between calls
   uint32_t* passed;       // [m_pairs] down-tile producers that have seen the block complete; zero between calls
   uint32_t* status;
+  uint64_t wait_ns;       // limit of every bounded wait
+  uint32_t extra;         // added to the target of every wait for other CTAs' arrivals (0 outside tests)
 };
 
 struct Tile {
@@ -91,7 +92,8 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p) {
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // Bounded wait until `*counter` has reached `target`.
-__device__ __forceinline__ bool wait_count(const uint32_t* counter, uint32_t target, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool wait_count(const uint32_t* counter, uint32_t target, volatile uint32_t* abort_flag,
+                                           uint64_t WAIT_NS) {
   if (ld_acquire_gpu(counter) >= target) return true;
   const uint64_t t0 = globaltimer_ns();
   uint32_t polls = 0;
@@ -124,6 +126,8 @@ tc_layer_kernel(const __grid_constant__ CUtensorMap tm_x,        // X   [n x d] 
   uint64_t* tempty_bar = tfull_bar + 2;                                  // used in the even CTA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  const ClockProbe probe = clock_probe_begin();
+  const uint64_t WAIT_NS = p.wait_ns;
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const uint32_t rank = cluster_ctarank();
@@ -178,7 +182,7 @@ tc_layer_kernel(const __grid_constant__ CUtensorMap tm_x,        // X   [n x d] 
         const uint32_t stage_tx = 2u * static_cast<uint32_t>(A_BYTES + half_rows * BK * 2);   // bytes of both CTAs
         if (t.is_down) {
           // H rows of this token block are complete once every gate|up tile of the block has arrived
-          if (!wait_count(p.done + t.m_pair, static_cast<uint32_t>(p.n1) * ARRIVALS_PER_GATEUP_TILE, abort_flag)) { ok = false; break; }
+          if (!wait_count(p.done + t.m_pair, static_cast<uint32_t>(p.n1) * ARRIVALS_PER_GATEUP_TILE + p.extra, abort_flag, WAIT_NS)) { ok = false; break; }
           fence_proxy_async_all();       // the TMA loads below must observe what that acquire made visible
           // the last of the 2 * n2 * ksplit producers of this block to get here re-arms the counters for the next call
           if (atomicAdd(p.passed + t.m_pair, 1u) == static_cast<uint32_t>(2 * p.n2 * p.ksplit - 1)) {
@@ -296,6 +300,7 @@ tc_layer_kernel(const __grid_constant__ CUtensorMap tm_x,        // X   [n x d] 
     tmem_dealloc_pair(tmem_base, TMEM_COLS);
   }
   if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, kStatusTimeout);
+  if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe_end(p.status, probe);
 }
 
 }  // namespace
@@ -499,6 +504,8 @@ cudaError_t launch_tc_layer(const TcLayerArgs& a, int num_sms, cudaStream_t st) 
   p.done = a.done;
   p.passed = a.passed;
   p.status = a.status;
+  p.wait_ns = a.wait.limit_ns;
+  p.extra = a.wait.extra_arrivals;
   const int pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;     // pairs without tiles have empty sequences
   return launch_pdl(tc_layer_kernel, dim3(2 * pairs), dim3(NUM_THREADS), SMEM_BYTES, st, a.tm_x, a.tm_wgu, a.tm_h_st, a.tm_h_ld,
                     a.tm_wdt, a.tm_y, p);

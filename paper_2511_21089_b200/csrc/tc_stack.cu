@@ -40,7 +40,6 @@ constexpr int SMEM_BYTES = BAR_OFFSET + 256 + 1024;
 static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 constexpr int ACC_STRIDE = 256;                      // TMEM columns per accumulator buffer
 constexpr int TMEM_COLS = 512;
-constexpr uint64_t WAIT_NS = 1000000000ull;
 constexpr int STACK_THREADS = 256;                   // producer, MMA, 4 epilogue and 2 norm warps
 constexpr uint32_t ARRIVALS_PER_ITEM = 8;            // 4 epilogue warps in each of the two CTAs
 constexpr int NORM_PARTS = kStackNormParts;          // norm items per 256-token block
@@ -61,6 +60,8 @@ struct StackParams {
   uint32_t* done_gu;      // [L x m_pairs] arrivals of gate|up tiles
   uint32_t* done_dn;      // [L x m_pairs] arrivals of down items
   uint32_t* status;
+  uint64_t wait_ns;       // limit of every bounded wait
+  uint32_t extra;         // added to the target of every wait for other CTAs' arrivals (0 outside tests)
 };
 
 struct Item {
@@ -83,7 +84,8 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p) {
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // Bounded wait until `*counter` has reached `target`.
-__device__ __forceinline__ bool wait_count(const uint32_t* counter, uint32_t target, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool wait_count(const uint32_t* counter, uint32_t target, volatile uint32_t* abort_flag,
+                                           uint64_t WAIT_NS) {
   if (ld_acquire_gpu(counter) >= target) return true;
   const uint64_t t0 = globaltimer_ns();
   uint32_t polls = 0;
@@ -161,6 +163,8 @@ tc_stack_kernel(const __grid_constant__ CUtensorMap tm_x,        // Xn  [n x d] 
   uint64_t* tempty_bar = tfull_bar + 2;                                  // used in the even CTA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  const ClockProbe probe = clock_probe_begin();
+  const uint64_t WAIT_NS = p.wait_ns;
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const uint32_t rank = cluster_ctarank();
@@ -222,7 +226,7 @@ tc_stack_kernel(const __grid_constant__ CUtensorMap tm_x,        // Xn  [n x d] 
         const uint32_t target = down ? static_cast<uint32_t>(L->n1) * ARRIVALS_PER_ITEM : NORM_PARTS * ARRIVALS_PER_NORM_ITEM;
         const bool known = t.m_pair < 64 && ((ready[down ? 1 : 0] >> t.m_pair) & 1u);
         if (!known) {
-          if (!wait_count(counter, target, abort_flag)) { ok = false; break; }
+          if (!wait_count(counter, target + p.extra, abort_flag, WAIT_NS)) { ok = false; break; }
           fence_proxy_async_all();       // the TMA loads below must observe what that acquire made visible
           if (t.m_pair < 64) ready[down ? 1 : 0] |= uint64_t(1) << t.m_pair;
         }
@@ -289,7 +293,7 @@ tc_stack_kernel(const __grid_constant__ CUtensorMap tm_x,        // Xn  [n x d] 
         // x rows of the block are final once every down item of the previous layer has added its part
         bool ok = true;
         if (lane == 0)
-          ok = wait_count(p.done_dn + cidx - p.m_pairs, static_cast<uint32_t>(p.n2 * p.layers[t.layer - 1].ksplit) * ARRIVALS_PER_ITEM, abort_flag);
+          ok = wait_count(p.done_dn + cidx - p.m_pairs, static_cast<uint32_t>(p.n2 * p.layers[t.layer - 1].ksplit) * ARRIVALS_PER_ITEM + p.extra, abort_flag, WAIT_NS);
         ok = __all_sync(0xFFFFFFFFu, ok);    // also orders every lane's reads after lane 0's acquire
         if (!ok) break;
       }
@@ -350,6 +354,7 @@ tc_stack_kernel(const __grid_constant__ CUtensorMap tm_x,        // Xn  [n x d] 
     tmem_dealloc_pair(tmem_base, TMEM_COLS);
   }
   if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, kStatusTimeout);
+  if (blockIdx.x == 0 && threadIdx.x == 0) clock_probe_end(p.status, probe);
 }
 
 inline int32_t encode_item(int type, int col, int m_pair) {
@@ -466,6 +471,8 @@ cudaError_t launch_tc_stack(const TcStackArgs& a, int num_sms, cudaStream_t st) 
   p.done_gu = a.counters + static_cast<int64_t>(a.n_layers) * p.m_pairs;
   p.done_dn = a.counters + 2 * static_cast<int64_t>(a.n_layers) * p.m_pairs;
   p.status = a.status;
+  p.wait_ns = a.wait.limit_ns;
+  p.extra = a.wait.extra_arrivals;
   const int pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
   return launch_pdl(tc_stack_kernel, dim3(2 * pairs), dim3(STACK_THREADS), SMEM_BYTES, st, a.tm_x, a.tm_y, p);
 }

@@ -14,7 +14,7 @@ import torch
 
 import oracle
 from paper_2511_21089_b200 import synth
-from tests.helpers import TOL_BF16, bits_of, dev_bf16, dev_f32, rel_err, stack_tolerance, stream_ptr
+from tests.helpers import TOL_BF16, bits_of, dev_bf16, dev_f32, rel_err, rms_err, stack_tolerance, stream_ptr
 
 pytestmark = pytest.mark.gpu
 
@@ -138,13 +138,18 @@ def test_config4_decode_stack(lib, llama_stack):
                                                return_layer_inputs=True)
             check_layers_one_by_one(lib, handles, range(L), inputs, ref, 64)
             check_layers_one_by_one(lib, handles, (0, L - 1), [v[:1] for v in inputs], ref[:1], 1)
+            # End to end over 32 layers: first-order sum of the per-layer allowances on the worst element
+            # (about 0.09 of RMS(x_out) here), 2e-2 on the bulk (RMS) of the error.
             tol = stack_tolerance(inputs, ref)
-            assert tol < 0.25
+            assert tol < 0.12
             for n in (1, 8, 32, 64):
                 xd = dev_f32(x[:n])
                 lib.mlpmoe_stack_forward(handles, xd, n, 1e-6, stream_ptr())
                 torch.cuda.synchronize()
-                assert rel_err(xd.cpu().numpy(), ref[:n]) <= tol, (K, n)
+                e_max, e_rms = rel_err(xd.cpu().numpy(), ref[:n]), rms_err(xd.cpu().numpy(), ref[:n])
+                print(f"config 4 end to end, K={K}, n={n}: max|delta|/RMS = {e_max:.4f} (bound {tol:.4f}), RMS(delta)/RMS = {e_rms:.5f}")
+                assert e_max <= tol, (K, n)
+                assert e_rms <= TOL_BF16, (K, n)
             assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
     finally:
         destroy(lib, handles)
@@ -174,8 +179,13 @@ def test_config5_prefill_sweep_corners(lib, llama_stack, B, n, ratio):
                                            return_layer_inputs=True)
         got = xd.cpu().numpy()
         assert np.isfinite(got).all()
-        assert rel_err(got[rows], ref) <= stack_tolerance(inputs, ref)
-        check_layers_one_by_one(lib, handles, (0, L // 2, L - 1), inputs, ref, n)
+        tol = stack_tolerance(inputs, ref)
+        e_max, e_rms = rel_err(got[rows], ref), rms_err(got[rows], ref)
+        print(f"config 5 end to end, B={B}, n={n}, ratio={ratio}: max|delta|/RMS = {e_max:.4f} (bound {tol:.4f}), RMS(delta)/RMS = {e_rms:.5f}")
+        assert tol < 0.12
+        assert e_max <= tol
+        assert e_rms <= TOL_BF16
+        check_layers_one_by_one(lib, handles, list(range(0, L, 4)) + [L - 1], inputs, ref, n)
         assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
     finally:
         destroy(lib, handles)

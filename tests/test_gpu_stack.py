@@ -7,7 +7,7 @@ import torch
 
 import oracle
 from paper_2511_21089_b200 import synth
-from tests.helpers import TOL_BF16, TOL_FP32, Case, dev_bf16, dev_f32, rel_err, stack_tolerance, stream_ptr
+from tests.helpers import TOL_BF16, TOL_FP32, Case, dev_bf16, dev_f32, layer_rms, rel_err, rms_err, stack_tolerance, stream_ptr
 
 pytestmark = pytest.mark.gpu
 
@@ -100,20 +100,68 @@ def test_config2_full_size_sampled_rows(lib):
         ref, inputs = oracle.stack_forward(x[rows], layers, bf16_activations=True, return_layer_inputs=True)
         got = xd.cpu().numpy()
         assert np.isfinite(got).all()
-        # end to end: per-layer allowances add up over the 24 layers (see stack_tolerance)
-        tol = stack_tolerance(inputs, ref)
-        assert tol < 0.2
-        assert rel_err(got[rows], ref) <= tol
-        # every 4th layer on its own, fed the oracle's input of that layer, at the layer tolerance
+        # End to end over 24 layers: the worst element sits at about 2e-2 RMS (bf16 rounding of H adds up like a
+        # random walk), so the bound is 3e-2 on the worst element and 2e-2 / 4 on the bulk (RMS) of the error.
+        e_max, e_rms = rel_err(got[rows], ref), rms_err(got[rows], ref)
+        print(f"config 2 end to end: max|delta|/RMS = {e_max:.4f}, RMS(delta)/RMS = {e_rms:.5f}, "
+              f"first-order bound {stack_tolerance(inputs, ref):.4f}")
+        assert e_max <= 3e-2
+        assert e_rms <= TOL_BF16 / 4
+        # every layer on its own, fed the oracle's input of that layer, at the layer tolerance
         xs = inputs + [ref]
-        for l in list(range(0, L, 4)) + [L - 1]:
+        worst = 0.0
+        for l in range(L):
             xin = np.zeros((n, d), dtype=np.float32)
             xin[:len(rows)] = xs[l].astype(np.float32)
             xin_d = dev_f32(xin)
             lib.mlpmoe_stack_forward(handles[l:l + 1], xin_d, n, 1e-6, stream_ptr())
             torch.cuda.synchronize()
             delta_got = xin_d.cpu().numpy()[:len(rows)].astype(np.float64) - xin[:len(rows)].astype(np.float64)
-            assert rel_err(delta_got, xs[l + 1] - xs[l]) <= TOL_BF16, l
+            e = rel_err(delta_got, xs[l + 1] - xs[l])
+            worst = max(worst, e)
+            assert e <= TOL_BF16, l
+        print(f"config 2 layer by layer: worst max|delta|/RMS(y_l) = {worst:.4f}")
+        assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
+    finally:
+        for h in handles[1:] + handles[:1]:
+            lib.mlpmoe_destroy(h)
+
+
+def test_two_full_width_layers_every_row(lib):
+    """What the one-launch prefill-stack kernel adds over a single layer, at full width and checked on
+    EVERY row: 2 layers of the Qwen shape over 4096 tokens = 16 token blocks, so the down items trail
+    their block's gate|up tiles by 7 blocks across the layer boundary, the norm warps race the GEMM
+    pipeline, and every (layer, block) dependency counter is in use.  A K slice dropped or added twice,
+    or a block normalised before its down items are in, moves whole rows by far more than the bound."""
+    cfg = synth.CONFIGS[2]
+    d, I, B, n, L = cfg["d_model"], cfg["d_inter"], cfg["B"], cfg["n"], 2
+    d_b = synth.equal_partition(I, B)
+    handles, layers = [], []
+    try:
+        for l in range(L):
+            bits = synth.layer_weights(2, l, d, I, 0.02, bf16=True)
+            keep = synth.keep_set((synth.BASE_SEED, 2, l, synth.T_KEEP), B, cfg["n_drop"])
+            dev = [dev_bf16(b) for b in bits]
+            h = lib.mlpmoe_create(d, I, d_b, dev[0], dev[1], dev[2], None, lib.MLPMOE_BF16, lib.MLPMOE_LAYOUT_PAPER, n, stream_ptr())
+            lib.mlpmoe_prune(h, keep, True, stream_ptr())
+            if handles:
+                lib.mlpmoe_share_workspace(h, handles[0])
+            handles.append(h)
+            layers.append((*[synth.bf16_bits_to_f32(b) for b in bits], d_b, oracle.prune_alpha([1.0] * B, keep)))
+        x = synth.tokens(2, n, d)
+        ref, inputs = oracle.stack_forward(x, layers, bf16_activations=True, return_layer_inputs=True)
+        bound = stack_tolerance(inputs, ref)           # first order: TOL_BF16 * (RMS(y_0) + RMS(y_1)) / RMS(x_out)
+        for rep in range(3):                           # arrival order differs from run to run
+            xd = dev_f32(x)
+            lib.mlpmoe_stack_forward(handles, xd, n, 1e-6, stream_ptr())
+            torch.cuda.synchronize()
+            got = xd.cpu().numpy()
+            e_max, e_rms = rel_err(got, ref), rms_err(got, ref)
+            print(f"2 Qwen layers, all {n} rows, run {rep}: max|delta|/RMS = {e_max:.5f} (bound {bound:.5f}), RMS(delta)/RMS = {e_rms:.6f}")
+            assert e_max <= bound
+            # measured against the layers' own contribution (what the kernel computes), the bulk of the error is tiny
+            y_got = got.astype(np.float64) - x
+            assert rms_err(y_got, ref - x) <= TOL_BF16 / 4
         assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
     finally:
         for h in handles[1:] + handles[:1]:

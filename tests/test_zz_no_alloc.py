@@ -47,9 +47,11 @@ def test_static_fade_matches_handle_fade_twice(lib, bf16):
             for b in range(len(d_b)):
                 slices.append(W[:, offs[b]:offs[b + 1]].contiguous())
                 ratios.append(s[b])
-        before = torch.cuda.memory_allocated()
+        # cudaMalloc inside the library would not show in torch's caching allocator: watch the device's free memory
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         lib.mlpmoe_fade_buffers_static(slices, ratios, dtype, stream_ptr())
-        assert torch.cuda.memory_allocated() == before
+        assert torch.cuda.mem_get_info()[0] >= free_before
         for k, (W, ref) in enumerate(((c.dev[0], ref_g), (c.dev[1], ref_u))):
             for b in range(len(d_b)):
                 got = slices[k * len(d_b) + b]
@@ -77,5 +79,11 @@ def test_static_fade_rejects_bad_arguments(lib):
         lib.mlpmoe_fade_buffers_static([x], [1.0], lib.MLPMOE_FP32, stream_ptr())
     assert e.value.status == lib.MLPMOE_ERR_BAD_SCHEDULE
     assert lib.lib.mlpmoe_fade_buffers_static(None, None, None, 3, 1, None) == lib.MLPMOE_ERR_INVALID_ARG
+    # a slice that is not aligned to its element size is refused on the host (nothing is launched)
+    for dtype, off in ((lib.MLPMOE_FP32, 2), (lib.MLPMOE_FP32, 1), (lib.MLPMOE_BF16, 1)):
+        ptrs = (ctypes.c_void_p * 1)(x.data_ptr() + off)
+        m = (ctypes.c_int64 * 1)(8)
+        s = (ctypes.c_double * 1)(0.5)
+        assert lib.lib.mlpmoe_fade_buffers_static(ptrs, m, s, 1, dtype, None) == lib.MLPMOE_ERR_INVALID_ARG
     lib.mlpmoe_fade_buffers_static([], [], lib.MLPMOE_FP32, stream_ptr())   # nothing to do
     assert float(x.abs().sum()) == 0.0
