@@ -165,11 +165,12 @@ def time_oracle(w, rows: int, n_layers: int, steps: int, warmup: int):
 
 
 def oracle_sample(w, arm: str):
-    """(rows, layers) of the CPU sample.  On Llama-shaped layers most of a pass is the oracle widening each
-    layer's weights to float64 (about 2 s per layer whatever the row count), so the sample is cut in layers:
-    the reference arm (steps + warm-up passes) takes 2 layers, the one-pass baseline of the default run 4."""
+    """(rows, layers) of the CPU sample.  On Llama-shaped layers a pass costs about 0.3 s per layer (much of it the
+    oracle widening the layer's weights to float64, whatever the row count): the one-pass baseline of the default
+    run takes 64 rows through the whole stack, the reference arm (steps + warm-up passes) 32 rows through the first
+    8 layers."""
     if w["d"] >= 4096:
-        return (32, min(2, w["L"])) if arm == "reference" else (64, min(4, w["L"]))
+        return (32, min(8, w["L"])) if arm == "reference" else (64, w["L"])
     return 256, w["L"]
 
 
