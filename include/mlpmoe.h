@@ -102,6 +102,21 @@ mlpmoe_status_t mlpmoe_share_workspace(mlpmoe_handle_t h, mlpmoe_handle_t donor)
 mlpmoe_status_t mlpmoe_fade(mlpmoe_handle_t h, const double* s, void* stream);
 
 /*
+ * Neuron-structured Fade: a LABELLED VARIANT of Fractal Fade, not the paper's definition (Section 3.2
+ * masks single weights, which saves no work on dense tensor-core tiles; Section 6.2 and Section 7
+ * name exactly that gap).  Same schedule, coarser grain: in every branch b with s_b > 0 the
+ * q_b = floor(s_b d_b) neurons with the smallest score are removed whole (their W_gate and W_up
+ * columns are zeroed; W_down is not touched), where
+ *     score_j = sum_k W_gate[k, j]^2 + sum_k W_up[k, j]^2
+ * is accumulated in float64 one term after the other in that order (products and sums rounded
+ * separately), and ties go to the lower neuron index first.  The removed neurons leave the schedule,
+ * so prefill and decode work shrink with them.  s as in mlpmoe_fade (NULL = s_b = 0.9 b / B, with
+ * q_b = (9 b d_b) div (10 B)).  Idempotent.  Allocates and frees temporary device memory;
+ * synchronises `stream`.
+ */
+mlpmoe_status_t mlpmoe_fade_structured(mlpmoe_handle_t h, const double* s, void* stream);
+
+/*
  * Compensated Branch Pruning (Section 3.3) with an arbitrary keep set:
  * alpha_b <- alpha_b(create) * sqrt(B / K) for kept branches (K = number kept;
  * factor 1 if `compensate` is 0) and 0 for the others, computed as

@@ -12,6 +12,9 @@ from .mlpmoe_oracle import (  # noqa: F401
     fade_position,
     fade_mask,
     fade,
+    neuron_scores,
+    fade_structured_count,
+    fade_structured,
     prune_alpha,
     first_k_keep,
     nnz_per_branch,

@@ -24,6 +24,9 @@ identity), brute-force scalar evaluation of tiny cases, hand-computed golden
 values, closed-form Fade zero counts and the paper's Table 1 / Table 2
 non-zero parameter counts, top-k-by-magnitude brute force for the Fade mask,
 exact sqrt(B/K) values and the variance-preservation claim of Section 3.3.
+fade_structured / neuron_scores are a labelled variant of this build (no passage
+of the paper defines them): pinned by a scalar brute force, the closed-form
+count of removed neurons and exact small-integer cases.
 The paper's perplexity and generation-time figures need trained checkpoints
 and an unpublished text mixture: parity unpinned for those (out of scope).
 """
@@ -167,6 +170,52 @@ def fade(W_gate, W_up, d_b: Sequence[int], s: Optional[Sequence] = None):
             sl = W[:, offs[b]:offs[b + 1]]
             keep = fade_mask(sl, s[b])
             sl *= keep.astype(W.dtype)
+    return Wg, Wu
+
+
+def neuron_scores(W_gate, W_up) -> np.ndarray:
+    """score_j = sum_k W_gate[k, j]^2 + sum_k W_up[k, j]^2 in float64, the terms added
+    one after the other in that order (the gate column first), so that any program
+    adding the same terms in the same order gets the same bits (the products of
+    float32 or bfloat16 values are exact in float64; the order fixes the sums)."""
+    g = np.asarray(W_gate).astype(np.float64)
+    u = np.asarray(W_up).astype(np.float64)
+    terms = np.concatenate([(g * g).T, (u * u).T], axis=1)        # [I, 2 d]: neuron j's terms in order
+    return np.cumsum(terms, axis=1)[:, -1]                        # a running sum is sequential by construction
+
+
+def fade_structured_count(s, d_b: int) -> int:
+    """q = floor(s * d_b) neurons leave a branch of width d_b (exact arithmetic)."""
+    p = _as_fraction(s) * d_b
+    return int(p.numerator // p.denominator)
+
+
+def fade_structured(W_gate, W_up, d_b: Sequence[int], s: Optional[Sequence] = None):
+    """Neuron-structured Fade, a labelled variant of Section 3.2 (NOT the paper's
+    definition, which masks single weights): with the same schedule s_b, branch b
+    loses its q_b = floor(s_b d_b) neurons of smallest neuron_scores, ties to the
+    lower index first; their W_gate and W_up columns become zero, W_down stays.
+    Returns masked copies."""
+    Wg = np.array(W_gate, copy=True)
+    Wu = np.array(W_up, copy=True)
+    B = len(d_b)
+    offs = branch_offsets(d_b, Wg.shape[1])
+    if s is None:
+        s = fade_schedule(B)
+    if len(s) != B:
+        raise ValueError("schedule must have one entry per branch")
+    score = neuron_scores(Wg, Wu)
+    for b in range(B):
+        sb = _as_fraction(s[b])
+        if not (0 <= sb < 1):
+            raise ValueError("sparsity ratio must lie in [0, 1)")
+        q = fade_structured_count(sb, int(d_b[b]))
+        if sb == 0 or q == 0:
+            continue
+        order = np.argsort(score[offs[b]:offs[b + 1]], kind="stable")      # ascending, ties to the lower index
+        gone = offs[b] + order[:q]
+        Wg[:, gone] = 0
+        Wu[:, gone] = 0
     return Wg, Wu
 
 

@@ -176,12 +176,8 @@ struct mlpmoe_layer_s {
   DecodeStackLayer* stack_dev = nullptr;                    // layer records of the persistent decode-stack kernel
   uint32_t* stack_counter = nullptr;                        // its grid-wide event counter
   std::vector<DecodeStackLayer> stack_host;                 // what stack_dev currently holds
-  // stage-tiled weight copies of the two decode-stack kernels (kDecTiledFused / kDecTiledStack), each built at the
-  // first set-up of its kernel after a (re)schedule, with the work split they were built for
-  void* dec_tiled[2] = {nullptr, nullptr};
-  int64_t dec_tiled_version[2] = {-1, -1};
-  int32_t* dec_bounds[2] = {nullptr, nullptr};              // device: [num_sms + 1] unit boundaries
-  int64_t* dec_a_off[2] = {nullptr, nullptr};               // device: [num_sms + 1] stream offsets
+  void* dec_tiled = nullptr;                                // stage-tiled weight copy of the fused few-token decode kernel,
+  int64_t dec_tiled_version = -1;                           //   built at the first such call after a (re)schedule
   // persistent prefill-stack kernel (buffers live in the first layer's handle, sized at the first call
   // with a new stack / token count)
   TcStackLayer* pstack_dev = nullptr;
@@ -243,8 +239,7 @@ void free_layer(mlpmoe_layer_s* h) {
   cudaFree(h->Wgu); cudaFree(h->WdT);
   cudaFree(h->scale); cudaFree(h->src_row); cudaFree(h->row_nnz);
   cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->block_done); cudaFree(h->tile_sched); cudaFree(h->stack_dev); cudaFree(h->stack_counter); cudaFree(h->status);
-  cudaFree(h->pstack_dev); cudaFree(h->pstack_items); cudaFree(h->pstack_counters);
-  for (int k = 0; k < 2; ++k) { cudaFree(h->dec_tiled[k]); cudaFree(h->dec_bounds[k]); cudaFree(h->dec_a_off[k]); }
+  cudaFree(h->pstack_dev); cudaFree(h->pstack_items); cudaFree(h->pstack_counters); cudaFree(h->dec_tiled);
   ws_release(h->ws);
   delete h;
 }
@@ -468,54 +463,41 @@ std::vector<int64_t> stack_key(const mlpmoe_handle_t* layers, int32_t n_layers, 
   return key;
 }
 
-// Set-up of the persistent decode kernels for this stack and token count: the stage-tiled weight copy of
-// the kernel that will run (allocated at the first decode set-up of a layer with that kernel, rebuilt after
-// a reschedule), the layer records and the token operand's tensor map.  MLPMOE_ERR_ALLOC if a copy cannot
-// be allocated (the caller then runs the stack layer by layer).
+// Set-up of the persistent decode kernels for this stack and token count: the stage-tiled weight copies
+// (allocated at the first decode set-up of a layer, rebuilt after a reschedule), the layer records and
+// the token operand's tensor map.
 mlpmoe_status_t plan_decode(const mlpmoe_handle_t* layers, int32_t n_layers, int64_t n, cudaStream_t st) {
   mlpmoe_layer_s* h0 = layers[0];
   const int npad = n <= 16 ? 16 : (n <= 32 ? 32 : 64);
-  const bool fused = n <= kDecodeFusedMaxTokens;
-  const int kind = fused ? kDecTiledFused : kDecTiledStack;
-  const int ctas = h0->num_sms;
-  std::vector<int32_t> bounds(static_cast<size_t>(ctas) + 1);
-  std::vector<int64_t> a_off(static_cast<size_t>(ctas) + 1);
-  for (int l = 0; l < n_layers; ++l) {
+  bool tiled = true;
+  for (int l = 0; tiled && l < n_layers; ++l) {
     mlpmoe_layer_s* h = layers[l];
-    if (h->dec_tiled[kind] != nullptr && h->dec_tiled_version[kind] == h->version) continue;
-    if (h->dec_tiled[kind] == nullptr) {
-      if (cudaMalloc(&h->dec_tiled[kind], decode_tiled_bytes(kind, h->Ipad_max, h->d)) != cudaSuccess ||
-          cudaMalloc(reinterpret_cast<void**>(&h->dec_bounds[kind]), sizeof(int32_t) * (ctas + 1)) != cudaSuccess ||
-          cudaMalloc(reinterpret_cast<void**>(&h->dec_a_off[kind]), sizeof(int64_t) * (ctas + 1)) != cudaSuccess) {
-        cudaGetLastError();
-        cudaFree(h->dec_tiled[kind]); cudaFree(h->dec_bounds[kind]); cudaFree(h->dec_a_off[kind]);
-        h->dec_tiled[kind] = nullptr; h->dec_bounds[kind] = nullptr; h->dec_a_off[kind] = nullptr;
-        return MLPMOE_ERR_ALLOC;
-      }
+    if (h->dec_tiled != nullptr && h->dec_tiled_version == h->version) continue;
+    if (h->dec_tiled == nullptr && cudaMalloc(&h->dec_tiled, decode_tiled_bytes(h->Ipad_max, h->d)) != cudaSuccess) {
+      cudaGetLastError();
+      h->dec_tiled = nullptr;
+      tiled = false;          // without memory for the copy the 14..64-token kernel reads the packed operands through tensor maps
+      break;
     }
-    decode_split(kind, h->Ipad, h->d, ctas, bounds.data(), a_off.data());
-    CK(cudaMemcpyAsync(h->dec_bounds[kind], bounds.data(), sizeof(int32_t) * (ctas + 1), cudaMemcpyHostToDevice, st));
-    CK(cudaMemcpyAsync(h->dec_a_off[kind], a_off.data(), sizeof(int64_t) * (ctas + 1), cudaMemcpyHostToDevice, st));
-    CK(launch_retile_decode(kind, h->Wgu, h->WdT, h->dec_tiled[kind], h->dec_bounds[kind], h->dec_a_off[kind], ctas, h->Ipad, h->d, st));
-    h->dec_tiled_version[kind] = h->version;
+    CK(launch_retile_decode(h->Wgu, h->WdT, h->dec_tiled, h->Ipad, h->d, st));
+    h->dec_tiled_version = h->version;
   }
   h0->stack_host.assign(static_cast<size_t>(n_layers), DecodeStackLayer());
   std::memset(h0->stack_host.data(), 0, sizeof(DecodeStackLayer) * h0->stack_host.size());
   for (int l = 0; l < n_layers; ++l) {
     mlpmoe_layer_s* h = layers[l];
     DecodeStackLayer& r = h0->stack_host[l];
+    r.tm_wgu = h->tm_wgu;
+    r.tm_wdt = h->tm_wdt256;
     if (!make_tmap(&r.tm_hd, h->ws->H, h->Ipad, n, h->Ipad, npad)) return MLPMOE_ERR_CUDA;
     r.scale = h->scale;
     r.Hd = static_cast<__nv_bfloat16*>(h->ws->H);
-    r.tiled = static_cast<const uint8_t*>(h->dec_tiled[kind]);
-    r.bounds = h->dec_bounds[kind];
-    r.a_off = h->dec_a_off[kind];
-    r.b_base = decode_tiled_b_base(h->Ipad, h->d);
+    r.tiled = tiled ? static_cast<const uint8_t*>(h->dec_tiled) : nullptr;
     r.Ipad = static_cast<int32_t>(h->Ipad);
   }
   CK(cudaMemcpyAsync(h0->stack_dev, h0->stack_host.data(), sizeof(DecodeStackLayer) * h0->stack_host.size(), cudaMemcpyHostToDevice, st));
   if (!make_tmap(&h0->plan_tm_x, h0->ws->xnorm, h0->d, n, h0->d, npad)) return MLPMOE_ERR_CUDA;
-  h0->plan_fused = fused;
+  h0->plan_fused = tiled && n <= kDecodeFusedMaxTokens;
   h0->plan_npad = npad;
   return MLPMOE_OK;
 }
@@ -595,10 +577,6 @@ mlpmoe_status_t plan_stack(const mlpmoe_handle_t* layers, int32_t n_layers, int6
   mlpmoe_status_t rc = MLPMOE_OK;
   if (kind == PLAN_DECODE) {
     rc = plan_decode(layers, n_layers, n, st);
-    if (rc == MLPMOE_ERR_ALLOC) {        // no memory for a stage-tiled copy: one pair of decode kernels per layer
-      kind = PLAN_PER_LAYER;
-      rc = MLPMOE_OK;
-    }
   } else if (kind == PLAN_PREFILL_STACK) {
     rc = plan_prefill_stack(layers, n_layers, n, st);
   } else if (h0->dtype == MLPMOE_BF16 && n > 128) {
@@ -806,6 +784,49 @@ mlpmoe_status_t mlpmoe_fade(mlpmoe_handle_t h, const double* s, void* stream) {
   }
   CK(launch_fade(segs.data(), static_cast<int>(segs.size()), h->fade_work, h->elem_size, st));
   CK(cudaStreamSynchronize(st));     // segs is host memory read by an async copy
+  return reschedule(h, st);
+}
+
+mlpmoe_status_t mlpmoe_fade_structured(mlpmoe_handle_t h, const double* s, void* stream) {
+  if (!h) return MLPMOE_ERR_INVALID_ARG;
+  if (s) {
+    for (int b = 0; b < h->B; ++b)
+      if (!(s[b] >= 0.0 && s[b] < 1.0)) return MLPMOE_ERR_BAD_SCHEDULE;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // scores of all neurons (device, float64, fixed summation order), then the selection on the host
+  double* score_dev = nullptr;
+  int32_t* rows_dev = nullptr;
+  if (cudaMalloc(reinterpret_cast<void**>(&score_dev), sizeof(double) * h->I) != cudaSuccess) { cudaGetLastError(); return MLPMOE_ERR_ALLOC; }
+  std::vector<double> score(static_cast<size_t>(h->I));
+  cudaError_t e = launch_neuron_scores(h->Wg_c, h->Wu_c, score_dev, h->I, h->d, h->elem_size, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(score.data(), score_dev, sizeof(double) * h->I, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  cudaFree(score_dev);
+  if (e != cudaSuccess) return MLPMOE_ERR_CUDA;
+  std::vector<int32_t> drop;
+  std::vector<int32_t> order;
+  for (int b = 0; b < h->B; ++b) {
+    if (s ? (s[b] == 0.0) : (b == 0)) continue;                   // the dense backbone / "leave untouched"
+    const int64_t m = h->d_b[b];
+    // q = floor(s_b * d_b) in exact arithmetic
+    const int64_t q = s ? fade_position_exact(s[b], m + 1)
+                        : static_cast<int64_t>((static_cast<__int128>(9) * b * m) / (static_cast<__int128>(10) * h->B));
+    if (q <= 0) continue;
+    order.resize(static_cast<size_t>(m));
+    for (int64_t i = 0; i < m; ++i) order[i] = static_cast<int32_t>(h->offs[b] + i);
+    // ascending score, ties to the lower index (stable): the first q go
+    std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return score[x] < score[y]; });
+    drop.insert(drop.end(), order.begin(), order.begin() + q);
+  }
+  if (!drop.empty()) {
+    if (cudaMalloc(reinterpret_cast<void**>(&rows_dev), sizeof(int32_t) * drop.size()) != cudaSuccess) { cudaGetLastError(); return MLPMOE_ERR_ALLOC; }
+    e = cudaMemcpyAsync(rows_dev, drop.data(), sizeof(int32_t) * drop.size(), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = launch_zero_rows(h->Wg_c, h->Wu_c, rows_dev, static_cast<int64_t>(drop.size()), h->d, h->elem_size, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cudaFree(rows_dev);
+    if (e != cudaSuccess) return MLPMOE_ERR_CUDA;
+  }
   return reschedule(h, st);
 }
 

@@ -1,38 +1,40 @@
-// Decode of a whole pre-norm stack (14 to 64 tokens) in ONE persistent, cooperatively launched
+// Decode of a whole pre-norm stack (n_tokens <= 64) in ONE persistent, cooperatively launched
 // kernel: x <- x + MLPMoE_l(RMSNorm(x)) for l = 0 .. L-1.  One CTA per SM; every CTA walks the same
 // static sequence of phases per layer
 //     N: RMSNorm of the token rows into the bf16 activation buffer
-//     A: gate|up, H = bf16(silu(G) * U * scale), for the CTA's own share of the neurons (Section 3.1)
+//     A: gate|up, H = bf16(silu(G) * U * scale), 128 neurons per work item      (Section 3.1)
 //     B: down + branch sum, 256 output columns per work item, K slices added straight into the
 //        fp32 stream x
 // separated by grid-wide events (one global arrival counter, bounded waits).  The producer warp
 // never stops at an event with an empty ring: weight tiles depend on no earlier phase, so it keeps
 // issuing them and only holds back the small activation tile of each stage until the event it
 // needs has passed.  HBM therefore keeps streaming weights across phase and layer boundaries.
-// Phase A deals the layer's neurons to the CTAs in equal contiguous shares of 16-neuron units
-// (decode_common.cuh), phase B its (256-column block, K-step) units in equal contiguous ranges, so
-// every SM streams the same share of the weights whatever survives pruning.  A stage holds up to
-// 256 weight rows x 64 K (gate and up rows of the same neurons in phase A, two neighbouring blocks
-// of output columns in phase B) next to one token tile; the weights come from a stage-tiled copy
-// (launch_retile_decode) by plain bulk copies, a CTA's stages of a phase being one contiguous run.
+// Both phases use the same stage: 256 weight rows x 64 K (two accumulators of 128 rows: gate and
+// up of the same neurons in phase A, two neighbouring blocks of output columns in phase B) next to
+// one token tile, so every stage carries 32 KB of weights.  Where the layers have a stage-tiled
+// copy (launch_retile_decode) the weights of a stage are one contiguous, ready-made shared-memory
+// image fetched by a plain bulk copy (2 to 4 % faster than the 256 row pieces of a tensor tile);
+// otherwise they come from the packed operands through tensor maps.
 //
 // Warp roles: warp 0 TMA producer, warp 1 TMEM owner + MMA issuer, warps 2..5 epilogue (and the
 // RMSNorm phase).  Weights sit on the 128-row side of the MMA, tokens on N = 16 / 32 / 64.
 #include <cuda_bf16.h>
 
-#include "decode_common.cuh"
+#include "internal.h"
+#include "ptx.cuh"
 
 namespace mlpmoe {
 namespace {
 
 using namespace ptx;
-using namespace dec;
 
+constexpr int BK = 64;
+constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
 constexpr int MAXN = kDecodeMaxTokens;
 constexpr int MAX_STAGES = 6;
-constexpr int W_BYTES = 256 * BK * 2;                 // weight bytes of a full stage (256 rows)
-// A stage slot is a full weight tile plus a token tile of npad rows; the ring takes as many slots as fit
+constexpr int W_BYTES = 256 * BK * 2;                 // 256 weight rows per stage in both phases
+// A stage is the weight tile plus a token tile of npad rows; the ring takes as many stages as fit
 // (6 for npad 16 and 32, 5 for npad 64), the barriers sit in front of it.
 constexpr int BAR_BYTES = 1024;
 constexpr int RING_BYTES = 216 * 1024;
@@ -43,6 +45,42 @@ __host__ __device__ constexpr int stages_for(int npad) {
   return RING_BYTES / stage_bytes_for(npad) < MAX_STAGES ? RING_BYTES / stage_bytes_for(npad) : MAX_STAGES;
 }
 constexpr uint32_t TMEM_COLS = 4 * MAXN;              // 2 buffers x (G | U)
+constexpr uint32_t ARRIVALS_PER_CTA = 1;              // one arrival per CTA and event, after its four epilogue warps have met
+constexpr int NORM_VEC = 8;                           // float4 per lane the RMSNorm phase keeps in registers
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// The four epilogue warps (threads 64..191) only.
+__device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Events are numbered in program order, 3 per layer (N, A, B), and each has its own arrival counter
+// (a CTA without work in a phase arrives at once, so one shared counter would let early arrivals
+// at later events stand in for missing arrivals at earlier ones).  Event e has happened once
+// counter[e] has reached arrivals_per_event.
+__device__ __forceinline__ bool event_passed(const uint32_t* counter, uint32_t target) {
+  return ld_acquire_u32(counter) >= target;
+}
+__device__ __forceinline__ bool event_wait(const uint32_t* counter, uint32_t target, volatile uint32_t* abort_flag,
+                                           uint64_t WAIT_NS) {
+  if (event_passed(counter, target)) return true;
+  const uint64_t t0 = globaltimer_ns();
+  uint32_t polls = 0;
+  while (true) {
+    if (event_passed(counter, target)) return true;
+    __nanosleep(64);
+    if ((++polls & 15u) == 0) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > WAIT_NS) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
 
 // Issues the loads of one accumulator's first npad columns; the values are valid after tmem_ld_wait().
 __device__ __forceinline__ void load_acc_async(uint32_t taddr, int npad, uint32_t (&v)[MAXN]) {
@@ -76,31 +114,25 @@ __device__ __forceinline__ int b_items(int cta, int ctas, int m_blocks, int kb2,
   return n;
 }
 
-// One CTA's weight stages of the whole stack in program order: per layer first phase A (its items,
-// all K-steps of each), then phase B (its items).  The producer walks the sequence.
+// One CTA's weight K-steps of the whole stack in program order: per layer first phase A (its
+// gate|up tiles, all K-steps of each), then phase B (its items).  The producer walks the
+// sequence.
 struct StepIter {
   const DecodeStackLayer* layers;
   int n_layers, cta, ctas, m_blocks, kb1;
-  int l, ph, idx, kb, nit;       // ph 0: idx = phase A item; ph 1: idx = phase B item
-  int a_lo, a_hi;                // phase A units of layer l
+  int l, ph, idx, kb, nit;       // ph 0: idx = gate|up tile; ph 1: idx = item number
   BItem it[4];
   bool done;
-  __device__ __forceinline__ int a_count() const { return (a_hi - a_lo + kDecMaxUnitsPerItem - 1) / kDecMaxUnitsPerItem; }
-  __device__ __forceinline__ int a_rows(int i) const {
-    const int left = a_hi - a_lo - i * kDecMaxUnitsPerItem;
-    return kDecUnit * (left < kDecMaxUnitsPerItem ? left : kDecMaxUnitsPerItem);
-  }
   __device__ __forceinline__ void settle() {      // moves to the first phase at or after (l, ph) that has work
     while (!done) {
+      const int Ipad = layers[l].Ipad;
       if (ph == 0) {
-        a_lo = layers[l].bounds[cta];
-        a_hi = layers[l].bounds[cta + 1];
-        idx = 0;
+        idx = cta;
         kb = 0;
-        if (a_hi > a_lo) return;
+        if (idx < Ipad / 128) return;
         ph = 1;
       }
-      nit = b_items(cta, ctas, m_blocks, layers[l].Ipad / BK, it);
+      nit = b_items(cta, ctas, m_blocks, Ipad / BK, it);
       idx = 0;
       if (nit > 0) { kb = it[0].kb_lo; return; }
       ph = 0;
@@ -109,28 +141,28 @@ struct StepIter {
   }
   __device__ __forceinline__ void init(const DecodeStackLayer* layers_, int n_layers_, int cta_, int ctas_, int m_blocks_, int kb1_) {
     layers = layers_; n_layers = n_layers_; cta = cta_; ctas = ctas_; m_blocks = m_blocks_; kb1 = kb1_;
-    l = 0; ph = 0; idx = 0; kb = 0; nit = 0; a_lo = a_hi = 0;
+    l = 0; ph = 0; idx = 0; kb = 0; nit = 0;
     done = n_layers == 0;
     settle();
   }
+  __device__ __forceinline__ const CUtensorMap* wmap() const { return ph == 0 ? &layers[l].tm_wgu : &layers[l].tm_wdt; }
+  __device__ __forceinline__ int wrow() const { return (ph == 0 ? idx : it[idx].m_blk) * 256; }
   __device__ __forceinline__ int event() const { return 3 * l + ph; }     // the event its activation tile waits for
-  // Weight bytes of the current stage and where they sit in the stage-tiled copy.
-  __device__ __forceinline__ uint32_t wbytes() const { return ph == 0 ? static_cast<uint32_t>(a_rows(idx)) * 256u : static_cast<uint32_t>(W_BYTES); }
+  // The same 256 x 64 weight tile in the stage-tiled copy (see launch_retile_decode): chunk kb of gate|up
+  // tile idx, or, for phase B, the chunk of output block m_blk and K-step kb = 2 * (gate|up tile) + half.
   __device__ __forceinline__ const uint8_t* wtiled() const {
-    const DecodeStackLayer& L = layers[l];
-    if (ph == 0) {
-      // the CTA's items follow one another, each with its kb1 stages of 256 * rows bytes
-      const int64_t before = static_cast<int64_t>(idx) * kDecMaxUnitsPerItem * kDecUnit * 256 * kb1;
-      return L.tiled + L.a_off[cta] + before + static_cast<int64_t>(kb) * a_rows(idx) * 256;
-    }
-    return L.tiled + L.b_base + (static_cast<int64_t>(it[idx].m_blk) * (L.Ipad / BK) + kb) * W_BYTES;
+    const int64_t cpt = kb1 + 2 * m_blocks;
+    const int64_t chunk = ph == 0 ? static_cast<int64_t>(idx) * cpt + kb
+                                  : static_cast<int64_t>(kb / 2) * cpt + kb1 + it[idx].m_blk * 2 + kb % 2;
+    return layers[l].tiled + chunk * W_BYTES;
   }
   __device__ __forceinline__ void advance() {
     ++kb;
     if (ph == 0) {
       if (kb < kb1) return;
+      idx += ctas;
       kb = 0;
-      if (++idx < a_count()) return;
+      if (idx < layers[l].Ipad / 128) return;
       ph = 1;
       settle();
     } else {
@@ -217,10 +249,10 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
         }
         if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, WAIT_NS)) { ok = false; break; }
         uint8_t* s = ring + stage * STAGE_BYTES;
-        const uint32_t wb = cur.wbytes();
-        mbar_expect_tx(&full_bar[stage], wb + act_bytes);
+        mbar_expect_tx(&full_bar[stage], W_BYTES + act_bytes);
         const int kc = cur.kb;     // every CTA walks K in the same order: staggered starts measured 3 % slower
-        bulk_load_1d(s, cur.wtiled(), wb, &full_bar[stage]);
+        if (layers[cur.l].tiled != nullptr) bulk_load_1d(s, cur.wtiled(), W_BYTES, &full_bar[stage]);
+        else tma_load_2d(s, cur.wmap(), kc * BK, cur.wrow(), &full_bar[stage]);
         if (gate_open) {
           tma_load_2d(s + W_BYTES, def_map, kc * BK, 0, &full_bar[stage]);
         } else {
@@ -238,7 +270,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
       const uint32_t idesc = make_idesc_bf16_f32(128, static_cast<uint32_t>(npad));
       int stage = 0, acc = 0; uint32_t phase = 0, acc_phase = 0; bool ok = true;
       // one work item: two accumulators of 128 weight rows each
-      auto run_item = [&](int kbs, int rows) -> bool {     // rows: weight rows per accumulator (second operand starts rows * 128 bytes in)
+      auto run_item = [&](int kbs) -> bool {
         if (!mbar_wait_bounded(&tempty_bar[acc], acc_phase ^ 1u, abort_flag, WAIT_NS)) return false;
         tc_fence_after();
         const uint32_t g_tmem = tmem_base + static_cast<uint32_t>(acc * 2 * MAXN);
@@ -247,7 +279,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
           tc_fence_after();
           const uint32_t s = smem_u32(ring + stage * STAGE_BYTES);
           const uint64_t w0 = make_desc_sw128_kmajor(s);
-          const uint64_t w1 = make_desc_sw128_kmajor(s + static_cast<uint32_t>(rows) * BK * 2);
+          const uint64_t w1 = make_desc_sw128_kmajor(s + 128 * BK * 2);
           const uint64_t xd = make_desc_sw128_kmajor(s + W_BYTES);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
@@ -265,11 +297,10 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
       };
       for (int l = 0; ok && l < n_layers; ++l) {
         const int Ipad = layers[l].Ipad;
-        const Items items(layers + l, cta);
-        for (int i = 0; ok && i < items.count(); ++i) ok = run_item(kb1, items.rows(i));
+        for (int tile = cta; ok && tile < Ipad / 128; tile += ctas) ok = run_item(kb1);
         BItem it[4];
         const int nit = b_items(cta, ctas, m_blocks, Ipad / BK, it);
-        for (int i = 0; ok && i < nit; ++i) ok = run_item(it[i].kb_hi - it[i].kb_lo, 128);
+        for (int i = 0; ok && i < nit; ++i) ok = run_item(it[i].kb_hi - it[i].kb_lo);
       }
     }
   }
@@ -278,10 +309,13 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
     const int quad = warp % 4;
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
-    auto arrive_event = [&](int e) {       // this warp's part of the phase is written and visible
-      __threadfence();
-      __syncwarp();
-      if (lane == 0) atomicAdd(event_counter + e, 1u);
+    // One arrival per CTA (592 arrivals on one counter took longer than the meeting of four warps): every
+    // thread makes its writes visible, the four warps meet, one thread arrives.  Called by all four warps
+    // also after a wait has given up, so that the named barrier stays balanced.
+    auto arrive_event = [&](int e) {
+      if (ok) __threadfence();
+      epilogue_bar_sync();
+      if (ok && quad == 0 && lane == 0) atomicAdd(event_counter + e, 1u);
     };
     auto wait_acc = [&]() -> bool {
       bool w = mbar_wait_bounded(&tfull_bar[acc], acc_phase, abort_flag, WAIT_NS);
@@ -306,18 +340,60 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
         bool w = event_wait(event_counter + 3 * l - 1, per_event, abort_flag, WAIT_NS);
         ok = __all_sync(0xFFFFFFFFu, w);
       }
-      for (int t = cta; t < n; t += ctas) norm_row(x, xnorm, t, d, eps, quad, lane, norm_part, ok);
-      if (ok) arrive_event(3 * l);                               // event N(l)
+      for (int t = cta; t < n; t += ctas) {
+        // each warp takes a quarter of the row, keeps it in registers, and the four partial sums of
+        // squares meet in shared memory
+        const float* row = x + static_cast<int64_t>(t) * d;
+        const int64_t q = (d / 4 + 3) / 4 * 4;                 // columns per warp, a multiple of 4
+        const int64_t c0 = static_cast<int64_t>(quad) * q, c1 = c0 + q < d ? c0 + q : d;
+        float4 v[NORM_VEC];
+        float ss = 0.f;
+        if (ok) {
+#pragma unroll
+          for (int i = 0; i < NORM_VEC; ++i) {
+            const int64_t k = c0 + (static_cast<int64_t>(i) * 32 + lane) * 4;
+            v[i] = k < c1 ? __ldcg(reinterpret_cast<const float4*>(row + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll
+          for (int i = 0; i < NORM_VEC; ++i) ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+          for (int64_t k = c0 + (static_cast<int64_t>(NORM_VEC) * 32 + lane) * 4; k < c1; k += 128) {   // rows wider than the register window
+            const float4 w4 = __ldcg(reinterpret_cast<const float4*>(row + k));
+            ss += w4.x * w4.x + w4.y * w4.y + w4.z * w4.z + w4.w * w4.w;
+          }
+          for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+        }
+        if (lane == 0) norm_part[quad] = ss;
+        epilogue_bar_sync();
+        const float total = norm_part[0] + norm_part[1] + norm_part[2] + norm_part[3];
+        epilogue_bar_sync();                                   // norm_part may be overwritten by the next row
+        if (ok) {
+          const float inv = 1.0f / sqrtf(total / static_cast<float>(d) + eps);
+          __nv_bfloat16* out = xnorm + static_cast<int64_t>(t) * d;
+          auto store4 = [&](int64_t k, const float4& f) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(f.x * inv, f.y * inv), hi = __floats2bfloat162_rn(f.z * inv, f.w * inv);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t*>(&lo);
+            pk.y = *reinterpret_cast<uint32_t*>(&hi);
+            *reinterpret_cast<uint2*>(out + k) = pk;
+          };
+#pragma unroll
+          for (int i = 0; i < NORM_VEC; ++i) {
+            const int64_t k = c0 + (static_cast<int64_t>(i) * 32 + lane) * 4;
+            if (k < c1) store4(k, v[i]);
+          }
+          for (int64_t k = c0 + (static_cast<int64_t>(NORM_VEC) * 32 + lane) * 4; k < c1; k += 128)
+            store4(k, __ldcg(reinterpret_cast<const float4*>(row + k)));
+        }
+      }
+      arrive_event(3 * l);                               // event N(l)
       // ---- phase A: Hd = bf16(silu(G) * U * scale)
       __nv_bfloat16* Hd = L->Hd;
-      const Items items(L, cta);
-      for (int item = 0; item < items.count(); ++item) {
+      for (int tile = cta; tile < Ipad / 128; tile += ctas) {
         if (ok && !wait_acc()) ok = false;
         if (!ok) continue;
         const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * 2 * MAXN) + (static_cast<uint32_t>(quad * 32) << 16);
-        const bool mine = quad * 32 + lane < items.rows(item);       // the accumulator lanes past the item's rows hold nothing
-        const int64_t j = static_cast<int64_t>(items.unit0(item)) * kDecUnit + quad * 32 + lane;
-        const float sc = mine ? L->scale[j] : 0.f;
+        const int64_t j = static_cast<int64_t>(tile) * 128 + quad * 32 + lane;
+        const float sc = L->scale[j];
 #pragma unroll
         for (int c = 0; c < MAXN; c += 32) {                   // 32 tokens at a time: gate and up columns together
           if (c < npad) {
@@ -333,7 +409,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               const int t = c + i;
-              if (t < n && mine) {
+              if (t < n) {
                 const float gv = __uint_as_float(g[i]);
                 Hd[static_cast<int64_t>(t) * Ipad + j] = __float2bfloat16_rn(__fdividef(gv, 1.0f + __expf(-gv)) * __uint_as_float(u[i]) * sc);
               }
@@ -341,7 +417,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
           }
         }
       }
-      if (ok) arrive_event(3 * l + 1);                           // event A(l)
+      arrive_event(3 * l + 1);                           // event A(l)
       // ---- phase B: every K slice adds its part into x
       BItem it[4];
       const int nit = b_items(cta, ctas, m_blocks, Ipad / BK, it);
@@ -363,7 +439,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
           }
         }
       }
-      if (ok) arrive_event(3 * l + 2);                           // event B(l)
+      arrive_event(3 * l + 2);                           // event B(l)
     }
   }
   __syncwarp();
@@ -382,7 +458,7 @@ cudaError_t decode_stack_init(int* max_ctas_per_sm) {
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(max_ctas_per_sm, decode_stack_kernel, NUM_THREADS, SMEM_BYTES);
 }
 
-// layers_dev: n_layers records in device memory (64-byte aligned; `tiled` in the kDecTiledStack layout).  event_counter: 3 * n_layers zeros.
+// layers_dev: n_layers records in device memory (64-byte aligned).  event_counter: 3 * n_layers zeros.
 cudaError_t launch_decode_stack(const DecodeStackLayer* layers_dev, int n_layers, const CUtensorMap& tm_x, float* x, void* xnorm,
                                 int64_t n, int64_t d, int npad, float eps, uint32_t* event_counter, uint32_t* status,
                                 int num_sms, const WaitCfg& wait, cudaStream_t st) {

@@ -67,6 +67,15 @@ cudaError_t launch_gather_down_t(const void* Wd_c, const int32_t* src_row, void*
 cudaError_t launch_row_nnz(const void* Wg_c, const void* Wu_c, const void* Wd_c, int32_t* out, int64_t I, int64_t d,
                            int elem_size, cudaStream_t st);
 
+// Three-way bf16 split of an fp32 matrix [rows x K] (row pitch src_pitch) into [rows x 3 Kp] bf16: segment s holds
+// piece s of every element (p0 + p1 + p2 = 24 significand bits of the value), K padded with zeros to Kp (multiple of 64).
+cudaError_t launch_split3(const float* src, void* dst, int64_t rows, int64_t K, int64_t Kp, int64_t src_pitch, cudaStream_t st);
+
+// Neuron-structured Fade variant: score[j] = sum of squares of neuron j's gate and up rows (float64, terms added
+// one after the other, gate row first); zero_rows clears the listed rows of both canonical matrices.
+cudaError_t launch_neuron_scores(const void* Wg_c, const void* Wu_c, double* score, int64_t I, int64_t d, int elem_size, cudaStream_t st);
+cudaError_t launch_zero_rows(void* A, void* B, const int32_t* rows_dev, int64_t n_rows, int64_t d, int elem_size, cudaStream_t st);
+
 // Fade: exact rank selection on magnitude bit patterns, then masking (Section 3.2).
 struct FadeSeg {
   void* base;      // first element of the slice (contiguous m elements)
@@ -77,27 +86,13 @@ struct FadeSeg {
 size_t fade_work_bytes(int nseg);
 cudaError_t launch_fade(const FadeSeg* segs_host, int nseg, void* work, int elem_size, cudaStream_t st);
 
-// Stage-tiled copies of the packed bf16 operands for the two decode-stack kernels: ready-made shared-memory
-// images of the kernels' stages, laid out so that everything one CTA streams for a layer is contiguous
-// (plain bulk copies; HBM serves long runs faster than 128-byte row pieces of a tensor tile).
-//   bounds[c] .. bounds[c + 1]: the 16-neuron units CTA c owns (c < ctas); a CTA's range is cut into items
-//   of at most 8 units.  For an item with r rows (neurons n0 ..):
-//   phase A stage kb (all layouts): r gate rows then r up rows x 64 K, 128-byte swizzle: 256 r bytes.
-//   kDecTiledFused: per item, its ceil(d / 64) phase A stages, then ceil(d / 128) phase B stages, each
-//     r / 16 sub-tiles of 128 output columns x 16 neurons (rows of 32 bytes, 32-byte swizzle): 256 r bytes.
-//   kDecTiledStack: all items' phase A stages, then at b_base the phase B region: chunk (block of 256 output
-//     columns, 64-wide K-step kb) at ((block * Ipad / 64) + kb) * 32 KB, 256 rows x 128 bytes, 128-byte swizzle.
-// Rows / columns past d are zero.
-enum { kDecTiledFused = 0, kDecTiledStack = 1 };
-constexpr int kDecUnit = 16;                 // neurons per unit of the decode kernels' work split
-constexpr int kDecMaxUnitsPerItem = 8;       // 128 weight rows: the M side of one MMA
-size_t decode_tiled_bytes(int kind, int64_t n_active_pad, int64_t d);
-int64_t decode_tiled_b_base(int64_t n_active_pad, int64_t d);     // kDecTiledStack: offset of the phase B region
-// bounds: [ctas + 1] units, a_off: [ctas + 1] bytes (host); equal shares of the n_active_pad / 16 units.
-void decode_split(int kind, int64_t n_active_pad, int64_t d, int ctas, int32_t* bounds, int64_t* a_off);
-// bounds_dev / a_off_dev: the same tables in device memory.
-cudaError_t launch_retile_decode(int kind, const void* Wgu, const void* WdT, void* tiled, const int32_t* bounds_dev,
-                                 const int64_t* a_off_dev, int ctas, int64_t n_active_pad, int64_t d, cudaStream_t st);
+// Stage-tiled copy of the packed bf16 operands for the fused few-token decode kernel: per tile of 128
+// compacted neurons one contiguous run of 32 KB chunks, each the 128-byte-swizzled shared-memory image
+// of one stage (256 rows x 64 K): first ceil(d / 64) chunks of Wgu rows [256 t, 256 t + 256) (K-step
+// after K-step), then per block of 256 output columns two chunks of WdT[block rows, the tile's
+// neurons 0..63 | 64..127].  Rows / columns past d are zero.
+size_t decode_tiled_bytes(int64_t n_active_pad, int64_t d);
+cudaError_t launch_retile_decode(const void* Wgu, const void* WdT, void* tiled, int64_t n_active_pad, int64_t d, cudaStream_t st);
 
 // r = x / sqrt(mean(x^2) + eps), out bf16 (elem_size 2) or fp32 (4).
 cudaError_t launch_rmsnorm(const float* x, void* r, int64_t n, int64_t d, float eps, int out_elem_size, cudaStream_t st);
@@ -118,6 +113,10 @@ struct TcGateUpArgs {
   void* H;              // [n x Ipad] bf16
   int64_t n, d, Ipad;
   uint32_t* status;
+  // split3 != 0 (fast fp32 mode): both operands are three-way bf16 splits [rows x 3 dp], dp = d rounded up to 64;
+  // the K loop runs the six piece products x0 w0, x0 w1, x0 w2, x1 w0, x1 w1, x2 w0, and H is written as the
+  // three-way split [n x 3 Ipad] of the fp32 value.
+  int split3 = 0;
 };
 struct TcDownArgs {
   CUtensorMap tm_h;     // H   [n x Ipad]         bf16, box 64 x 128
@@ -127,6 +126,7 @@ struct TcDownArgs {
   int y_bf16;
   int64_t n, d, Ipad;
   uint32_t* status;
+  int split3 = 0;       // fast fp32 mode: H and WdT are three-way splits [rows x 3 Ipad]; six piece products
 };
 cudaError_t launch_tc_gateup(const TcGateUpArgs& a, int num_sms, cudaStream_t st);
 cudaError_t launch_tc_down(const TcDownArgs& a, int num_sms, cudaStream_t st);
@@ -221,19 +221,18 @@ cudaError_t launch_decode_down(const DecodeArgs& a, int num_sms, cudaStream_t st
 cudaError_t decode_init();
 
 // ----------------------------------------------------------- decode_stack.cu --
-// One record per layer of a decode stack, read by the persistent stack kernels from device memory.
+// One record per layer of a decode stack, read by the persistent stack kernel from device memory.
 struct alignas(64) DecodeStackLayer {
-  CUtensorMap tm_hd;       // Hd  [n x Ipad]    box 64 x npad (token operand of the 14..64-token kernel's phase B)
-  const float* scale;      // [Ipad]
-  __nv_bfloat16* Hd;       // [n x Ipad]
-  const uint8_t* tiled;    // the launching kernel's stage-tiled weight copy
-  const int32_t* bounds;   // [ctas + 1] unit boundaries of the CTAs' phase A ranges
-  const int64_t* a_off;    // [ctas + 1] byte offset of each CTA's stream in `tiled`
-  int64_t b_base;          // kDecTiledStack: byte offset of the phase B region in `tiled`
+  CUtensorMap tm_wgu;    // Wgu [2 Ipad x d]  box 64 x 256
+  CUtensorMap tm_wdt;    // WdT [d x Ipad]    box 64 x 256
+  CUtensorMap tm_hd;     // Hd  [n x Ipad]    box 64 x npad
+  const float* scale;    // [Ipad]
+  __nv_bfloat16* Hd;     // [n x Ipad]
+  const uint8_t* tiled;  // stage-tiled weight copy of the fused few-token kernel (decode_tiled_bytes), else null
   int32_t Ipad;
-  int32_t pad_[3];
+  int32_t pad_[9];
 };
-static_assert(sizeof(DecodeStackLayer) == 192, "record layout");
+static_assert(sizeof(DecodeStackLayer) == 448, "record layout");
 cudaError_t decode_stack_init(int* max_ctas_per_sm);
 cudaError_t launch_decode_stack(const DecodeStackLayer* layers_dev, int n_layers, const CUtensorMap& tm_x, float* x, void* xnorm,
                                 int64_t n, int64_t d, int npad, float eps, uint32_t* event_counter, uint32_t* status,
@@ -241,7 +240,7 @@ cudaError_t launch_decode_stack(const DecodeStackLayer* layers_dev, int n_layers
 
 // ----------------------------------------------------------- decode_fused.cu --
 // Decode stack for at most kDecodeFusedMaxTokens tokens: both GEMMs of a layer on the CTA that owns the neurons.
-constexpr int kDecodeFusedMaxTokens = 13;   // above, the partial sums per CTA (fp32 atomics) cost more than the dependency saved (measured: even at 14)
+constexpr int kDecodeFusedMaxTokens = 13;   // above, the partial sums per tile (fp32 atomics) cost more than the dependency saved (measured: even at 14)
 cudaError_t decode_fused_init(int* max_ctas_per_sm);
 cudaError_t launch_decode_fused(const DecodeStackLayer* layers_dev, int n_layers, const CUtensorMap& tm_x, float* x, void* xnorm,
                                 int64_t n, int64_t d, float eps, uint32_t* event_counter, uint32_t* status, int num_sms,

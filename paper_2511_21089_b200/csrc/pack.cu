@@ -60,62 +60,89 @@ __global__ void gather_down_t_kernel(const T* __restrict__ Wd_c, const int32_t* 
   }
 }
 
-// ------------------------------------------ stage-tiled copies for decode ---
-// One thread per 16-byte piece (8 bf16) of the destination; layouts in internal.h.
-// Packed gate|up operand: neuron j's gate row is row (j / 128) * 256 + j % 128, its up row 128 further.
-__device__ __forceinline__ uint4 load_gateup_piece(const uint4* __restrict__ Wgu, int64_t j, int proj, int64_t k, int64_t d) {
-  if (k >= d) return make_uint4(0, 0, 0, 0);
-  const int64_t row = (j / kGroup) * (2 * kGroup) + proj * kGroup + j % kGroup;
-  return Wgu[(row * d + k) / 8];
-}
-
-// Phase A stages of every item of CTA blockIdx.y (grid.x strides over the CTA's pieces), and for the fused
-// layout the item's phase B stages behind them.
-__global__ void retile_items_kernel(int kind, const uint4* __restrict__ Wgu, const uint4* __restrict__ WdT, uint8_t* __restrict__ out,
-                                    const int32_t* __restrict__ bounds, const int64_t* __restrict__ a_off, int64_t Ipad, int64_t d) {
-  const int cta = blockIdx.y;
-  const int lo = bounds[cta], hi = bounds[cta + 1];
-  const int kb1 = static_cast<int>((d + 63) / 64), n_mb = static_cast<int>((d + 127) / 128);
-  const int64_t stages_per_item = kb1 + (kind == kDecTiledFused ? n_mb : 0);
-  int64_t item_base = a_off[cta];
-  for (int u0 = lo; u0 < hi; u0 += kDecMaxUnitsPerItem) {
-    const int r = kDecUnit * ((hi - u0) < kDecMaxUnitsPerItem ? (hi - u0) : kDecMaxUnitsPerItem);
-    const int64_t n0 = static_cast<int64_t>(u0) * kDecUnit;
-    const int64_t pieces_per_stage = 16 * r;                       // 256 r bytes
-    const int64_t pieces = pieces_per_stage * stages_per_item;
-    for (int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; q < pieces; q += static_cast<int64_t>(gridDim.x) * blockDim.x) {
-      const int64_t stage = q / pieces_per_stage;
-      const int p = static_cast<int>(q % pieces_per_stage);
-      uint4 v;
-      int64_t dst;                                                 // piece position inside the stage
-      if (stage < kb1) {
-        const int R = p / 8, c = p % 8;                            // row of the stage (gate rows, then up rows), piece of the row
-        v = load_gateup_piece(Wgu, n0 + R % r, R / r, stage * 64 + c * 8, d);
-        dst = R * 8 + (c ^ (R & 7));                               // 128-byte swizzle
-      } else {
-        const int64_t mb = stage - kb1;
-        const int k16 = p / 256, m = (p % 256) / 2, c = p % 2;     // sub-tile, output column of the block, piece of the 32-byte row
-        const int64_t col = mb * 128 + m;
-        v = col < d ? WdT[(col * Ipad + n0 + k16 * 16 + c * 8) / 8] : make_uint4(0, 0, 0, 0);
-        dst = static_cast<int64_t>(k16) * 256 + m * 2 + (c ^ ((m >> 2) & 1));   // 32-byte swizzle
-      }
-      reinterpret_cast<uint4*>(out + item_base)[stage * pieces_per_stage + dst] = v;
-    }
-    item_base += pieces * 16;
-  }
-}
-
-// Phase B region of the stack layout: chunk (block of 256 output columns, K-step) = 256 rows x 128 bytes.
-__global__ void retile_down_chunks_kernel(const uint4* __restrict__ WdT, uint4* __restrict__ out, int64_t Ipad, int64_t d, int64_t total) {
+// ------------------------------------------- stage-tiled copy for decode ---
+// One thread per 16-byte piece of the destination.  A chunk is 256 rows of 128 bytes; piece c of row r
+// goes to piece position c ^ (r % 8) of that row (the 128-byte swizzle of the shared-memory tiles).
+__global__ void retile_decode_kernel(const uint4* __restrict__ Wgu, const uint4* __restrict__ WdT, uint4* __restrict__ out,
+                                     int64_t Ipad, int64_t d, int kb1, int m_blocks, int64_t total) {
   const int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (q >= total) return;
+  const int chunks_per_tile = kb1 + 2 * m_blocks;
   const int c = static_cast<int>(q % 8), r = static_cast<int>((q / 8) % 256);
-  const int64_t chunk = q / 2048;
-  const int64_t kb2 = Ipad / 64;
-  const int64_t blk = chunk / kb2, kb = chunk % kb2;
-  const int64_t col = blk * 256 + r;
-  const uint4 v = col < d ? WdT[(col * Ipad + kb * 64 + c * 8) / 8] : make_uint4(0, 0, 0, 0);
-  out[chunk * 2048 + r * 8 + (c ^ (r & 7))] = v;
+  const int64_t chunk_id = q / 2048;
+  const int chunk = static_cast<int>(chunk_id % chunks_per_tile);
+  const int64_t tile = chunk_id / chunks_per_tile;
+  uint4 v = make_uint4(0, 0, 0, 0);
+  if (chunk < kb1) {
+    const int64_t col = static_cast<int64_t>(chunk) * 64 + c * 8;                 // K coordinate (elements)
+    if (col < d) v = Wgu[((tile * 256 + r) * d + col) / 8];
+  } else {
+    const int blk = (chunk - kb1) / 2, ks = (chunk - kb1) % 2;
+    const int64_t row = static_cast<int64_t>(blk) * 256 + r;                      // output column of the layer
+    if (row < d) v = WdT[(row * Ipad + tile * 128 + ks * 64 + c * 8) / 8];
+  }
+  out[chunk_id * 2048 + r * 8 + (c ^ (r & 7))] = v;
+}
+
+// ------------------------------------------------ three-way bf16 split -------
+// dst[r][s * Kp + k] = piece s of src[r][k] (s = 0, 1, 2; zero for K <= k < Kp), where
+//   p0 = bf16(v), p1 = bf16(v - p0), p2 = bf16(v - p0 - p1)      (differences exact in fp32)
+// so that p0 + p1 + p2 carries 24 significand bits of v.  One thread per 8 elements of a row.
+__global__ void split3_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t rows, int64_t K, int64_t Kp,
+                              int64_t src_pitch) {
+  const int64_t chunks = Kp / 8;
+  const int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (q >= rows * chunks) return;
+  const int64_t r = q / chunks, k0 = (q % chunks) * 8;
+  __nv_bfloat16 p[3][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float v = k0 + i < K ? src[r * src_pitch + k0 + i] : 0.f;
+    const __nv_bfloat16 a = __float2bfloat16_rn(v);
+    const float r1 = v - __bfloat162float(a);
+    const __nv_bfloat16 b = __float2bfloat16_rn(r1);
+    const __nv_bfloat16 c = __float2bfloat16_rn(r1 - __bfloat162float(b));
+    p[0][i] = a; p[1][i] = b; p[2][i] = c;
+  }
+#pragma unroll
+  for (int sgm = 0; sgm < 3; ++sgm)
+    *reinterpret_cast<uint4*>(dst + r * 3 * Kp + sgm * Kp + k0) = *reinterpret_cast<const uint4*>(p[sgm]);
+}
+
+// ------------------------------------------- neuron scores / row zeroing ----
+// score[j] = sum_k Wg_c[j][k]^2 + sum_k Wu_c[j][k]^2 in float64, accumulated one term after the other in
+// that order (gate row first) with separately rounded multiply and add, so that a host program adding the
+// same terms in the same order gets the same bits.  One thread per neuron (a set-up kernel).
+template <typename T>
+__device__ __forceinline__ double widen(T v);
+template <>
+__device__ __forceinline__ double widen<uint16_t>(uint16_t v) { return static_cast<double>(__uint_as_float(static_cast<uint32_t>(v) << 16)); }
+template <>
+__device__ __forceinline__ double widen<uint32_t>(uint32_t v) { return static_cast<double>(__uint_as_float(v)); }
+
+template <typename T>
+__global__ void neuron_score_kernel(const T* __restrict__ Wg_c, const T* __restrict__ Wu_c, double* __restrict__ score, int64_t I, int64_t d) {
+  const int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (j >= I) return;
+  double acc = 0.0;
+  for (int which = 0; which < 2; ++which) {
+    const T* row = (which == 0 ? Wg_c : Wu_c) + j * d;
+    for (int64_t k = 0; k < d; ++k) {
+      const double w = widen<T>(row[k]);
+      acc = __dadd_rn(acc, __dmul_rn(w, w));
+    }
+  }
+  score[j] = acc;
+}
+
+// Zeroes rows rows[i] (i < n_rows) of the two [I x d] matrices; one block per row.
+template <typename T>
+__global__ void zero_rows_kernel(T* __restrict__ A, T* __restrict__ B, const int32_t* __restrict__ rows, int64_t d) {
+  const int64_t j = rows[blockIdx.x];
+  for (int64_t k = threadIdx.x; k < d; k += blockDim.x) {
+    A[j * d + k] = 0;
+    B[j * d + k] = 0;
+  }
 }
 
 // ------------------------------------------------------------ row nnz -------
@@ -357,33 +384,42 @@ cudaError_t launch_row_nnz(const void* Wg_c, const void* Wu_c, const void* Wd_c,
   return cudaGetLastError();
 }
 
-int64_t decode_tiled_b_base(int64_t n_active_pad, int64_t d) { return n_active_pad * 256 * ((d + 63) / 64); }
-
-size_t decode_tiled_bytes(int kind, int64_t n_active_pad, int64_t d) {
-  if (kind == kDecTiledFused) return static_cast<size_t>(n_active_pad * 256 * ((d + 63) / 64 + (d + 127) / 128));
-  return static_cast<size_t>(decode_tiled_b_base(n_active_pad, d) + ((d + 255) / 256) * (n_active_pad / 64) * 32768);
+size_t decode_tiled_bytes(int64_t n_active_pad, int64_t d) {
+  const int64_t chunks_per_tile = (d + 63) / 64 + 2 * ((d + 255) / 256);
+  return static_cast<size_t>(n_active_pad / 128 * chunks_per_tile) * 32768;
 }
 
-void decode_split(int kind, int64_t n_active_pad, int64_t d, int ctas, int32_t* bounds, int64_t* a_off) {
-  const int64_t units = n_active_pad / kDecUnit;
-  const int64_t stages = (d + 63) / 64 + (kind == kDecTiledFused ? (d + 127) / 128 : 0);
-  for (int c = 0; c <= ctas; ++c) {
-    bounds[c] = static_cast<int32_t>(units * c / ctas);
-    a_off[c] = static_cast<int64_t>(bounds[c]) * kDecUnit * 256 * stages;
-  }
+cudaError_t launch_retile_decode(const void* Wgu, const void* WdT, void* tiled, int64_t n_active_pad, int64_t d, cudaStream_t st) {
+  const int64_t total = static_cast<int64_t>(decode_tiled_bytes(n_active_pad, d) / 16);
+  if (total == 0) return cudaSuccess;
+  retile_decode_kernel<<<cdiv(total, 256), 256, 0, st>>>(static_cast<const uint4*>(Wgu), static_cast<const uint4*>(WdT),
+                                                        static_cast<uint4*>(tiled), n_active_pad, d,
+                                                        static_cast<int>((d + 63) / 64), static_cast<int>((d + 255) / 256), total);
+  return cudaGetLastError();
 }
 
-cudaError_t launch_retile_decode(int kind, const void* Wgu, const void* WdT, void* tiled, const int32_t* bounds_dev,
-                                 const int64_t* a_off_dev, int ctas, int64_t n_active_pad, int64_t d, cudaStream_t st) {
-  if (n_active_pad == 0 || ctas <= 0) return cudaSuccess;
-  retile_items_kernel<<<dim3(64, ctas), 256, 0, st>>>(kind, static_cast<const uint4*>(Wgu), static_cast<const uint4*>(WdT),
-                                                      static_cast<uint8_t*>(tiled), bounds_dev, a_off_dev, n_active_pad, d);
-  if (kind == kDecTiledStack) {
-    const int64_t total = ((d + 255) / 256) * (n_active_pad / 64) * 2048;
-    retile_down_chunks_kernel<<<cdiv(total, 256), 256, 0, st>>>(
-        static_cast<const uint4*>(WdT), reinterpret_cast<uint4*>(static_cast<uint8_t*>(tiled) + decode_tiled_b_base(n_active_pad, d)),
-        n_active_pad, d, total);
-  }
+cudaError_t launch_split3(const float* src, void* dst, int64_t rows, int64_t K, int64_t Kp, int64_t src_pitch, cudaStream_t st) {
+  if (rows == 0) return cudaSuccess;
+  const int64_t total = rows * (Kp / 8);
+  split3_kernel<<<cdiv(total, 256), 256, 0, st>>>(src, static_cast<__nv_bfloat16*>(dst), rows, K, Kp, src_pitch);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_neuron_scores(const void* Wg_c, const void* Wu_c, double* score, int64_t I, int64_t d, int elem_size, cudaStream_t st) {
+  if (I == 0) return cudaSuccess;
+  if (elem_size == 2)
+    neuron_score_kernel<uint16_t><<<cdiv(I, 64), 64, 0, st>>>(static_cast<const uint16_t*>(Wg_c), static_cast<const uint16_t*>(Wu_c), score, I, d);
+  else
+    neuron_score_kernel<uint32_t><<<cdiv(I, 64), 64, 0, st>>>(static_cast<const uint32_t*>(Wg_c), static_cast<const uint32_t*>(Wu_c), score, I, d);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_zero_rows(void* A, void* B, const int32_t* rows_dev, int64_t n_rows, int64_t d, int elem_size, cudaStream_t st) {
+  if (n_rows == 0) return cudaSuccess;
+  if (elem_size == 2)
+    zero_rows_kernel<uint16_t><<<static_cast<unsigned>(n_rows), 256, 0, st>>>(static_cast<uint16_t*>(A), static_cast<uint16_t*>(B), rows_dev, d);
+  else
+    zero_rows_kernel<uint32_t><<<static_cast<unsigned>(n_rows), 256, 0, st>>>(static_cast<uint32_t*>(A), static_cast<uint32_t*>(B), rows_dev, d);
   return cudaGetLastError();
 }
 

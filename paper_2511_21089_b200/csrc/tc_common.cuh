@@ -14,7 +14,7 @@ constexpr int BK = 64;         // K elements per stage: one 128-byte swizzled ro
 constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
 
-enum { EPI_SWIGLU = 0, EPI_OUT = 1 };
+enum { EPI_SWIGLU = 0, EPI_OUT = 1, EPI_SWIGLU_SPLIT3 = 2 };
 
 struct EpiArgs {
   const float* scale;   // EPI_SWIGLU: per-neuron scale (effective alpha of the neuron's branch)
@@ -63,6 +63,47 @@ __device__ __forceinline__ void epilogue_swiglu(uint32_t taddr, const EpiArgs& e
       uint4* dst = reinterpret_cast<uint4*>(H + row * ep.ld + col0);
 #pragma unroll
       for (int v = 0; v < 4; ++v) dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+    }
+  }
+}
+
+// As epilogue_swiglu with the fp32 value h = silu(gate) * up * scale (accurate exp) written as its three-way
+// bf16 split: piece s of H[row, j] goes to column s * ep.cols + j of a row of 3 * ep.cols (= ep.ld) elements.
+__device__ __forceinline__ void epilogue_swiglu_split3(uint32_t taddr, const EpiArgs& ep, int64_t row, int64_t neuron0, int half) {
+  __nv_bfloat16* H = static_cast<__nv_bfloat16*>(ep.out);
+#pragma unroll 1
+  for (int c = 0; c < half; c += 16) {
+    uint32_t g[16], u[16];
+    ptx::tmem_ld_32x16(taddr + c, g);
+    ptx::tmem_ld_32x16(taddr + half + c, u);
+    ptx::tmem_ld_wait();
+    const int64_t col0 = neuron0 + c;
+    uint32_t pk[3][8];
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) {
+      __nv_bfloat16 p[3][2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float gv = __uint_as_float(g[i + e]);
+        const float h = gv / (1.0f + expf(-gv)) * __uint_as_float(u[i + e]) * __ldg(ep.scale + col0 + i + e);
+        const __nv_bfloat16 a = __float2bfloat16_rn(h);
+        const float r1 = h - __bfloat162float(a);
+        const __nv_bfloat16 b = __float2bfloat16_rn(r1);
+        p[0][e] = a; p[1][e] = b; p[2][e] = __float2bfloat16_rn(r1 - __bfloat162float(b));
+      }
+#pragma unroll
+      for (int s = 0; s < 3; ++s) {
+        __nv_bfloat162 v2(p[s][0], p[s][1]);
+        pk[s][i / 2] = *reinterpret_cast<uint32_t*>(&v2);
+      }
+    }
+    if (row < ep.rows) {
+#pragma unroll
+      for (int s = 0; s < 3; ++s) {
+        uint4* dst = reinterpret_cast<uint4*>(H + row * ep.ld + s * ep.cols + col0);
+        dst[0] = make_uint4(pk[s][0], pk[s][1], pk[s][2], pk[s][3]);
+        dst[1] = make_uint4(pk[s][4], pk[s][5], pk[s][6], pk[s][7]);
+      }
     }
   }
 }

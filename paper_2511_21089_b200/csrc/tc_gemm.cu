@@ -32,7 +32,10 @@ struct Cfg {
 template <int BN, int STAGES, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const EpiArgs ep,
-               int num_m_blocks, int num_n_blocks, int num_k_blocks) {
+               int num_m_blocks, int num_n_blocks, int num_k_blocks, int kseg) {
+  // K loop over num_k_blocks = terms * kseg blocks of 64: term t multiplies segment a_seg(t) of A's row by segment
+  // b_seg(t) of B's row.  One term (kseg = num_k_blocks) is the plain product; the six terms of the fast fp32
+  // mode pair the three-way splits of both operands as (0,0) (0,1) (0,2) (1,0) (1,1) (2,0).
   using C = Cfg<BN, STAGES>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -83,8 +86,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           if (!mbar_wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + stage * C::STAGE_BYTES;
           mbar_expect_tx(&full_bar[stage], C::STAGE_BYTES);
-          tma_load_2d(sa, &tm_a, kb * BK, m_blk * BM, &full_bar[stage]);
-          tma_load_2d(sa + C::A_BYTES, &tm_b, kb * BK, n_blk * BN, &full_bar[stage]);
+          const int term = kb / kseg, r = kb % kseg;
+          const int a_seg = term < 3 ? 0 : (term < 5 ? 1 : 2), b_seg = term < 3 ? term : (term < 5 ? term - 3 : 0);
+          tma_load_2d(sa, &tm_a, (a_seg * kseg + r) * BK, m_blk * BM, &full_bar[stage]);
+          tma_load_2d(sa + C::A_BYTES, &tm_b, (b_seg * kseg + r) * BK, n_blk * BN, &full_bar[stage]);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -140,6 +145,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * BN) + (static_cast<uint32_t>(quad * 32) << 16);
       if (EPI == EPI_SWIGLU)
         epilogue_swiglu(taddr, ep, row, static_cast<int64_t>(n_blk) * (BN / 2), BN / 2);
+      else if (EPI == EPI_SWIGLU_SPLIT3)
+        epilogue_swiglu_split3(taddr, ep, row, static_cast<int64_t>(n_blk) * (BN / 2), BN / 2);
       else
         epilogue_out(taddr, ep, row, static_cast<int64_t>(n_blk) * BN, BN);
       tc_fence_before();
@@ -169,6 +176,9 @@ cudaError_t tc_gemm_init() {
   cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<GU_BN, GU_STAGES, EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        Cfg<GU_BN, GU_STAGES>::SMEM_BYTES);
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(tc_gemm_kernel<GU_BN, GU_STAGES, EPI_SWIGLU_SPLIT3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           Cfg<GU_BN, GU_STAGES>::SMEM_BYTES);
+  if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(tc_gemm_kernel<DN_BN, DN_STAGES, EPI_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               Cfg<DN_BN, DN_STAGES>::SMEM_BYTES);
 }
@@ -183,12 +193,15 @@ cudaError_t launch_tc_gateup(const TcGateUpArgs& a, int num_sms, cudaStream_t st
   ep.out = a.H;
   ep.rows = a.n;
   ep.cols = a.Ipad;
-  ep.ld = a.Ipad;
+  ep.ld = a.split3 ? 3 * a.Ipad : a.Ipad;
   ep.status = a.status;
   const int tiles = m_blocks * n_blocks;
   const int grid = tiles < num_sms ? tiles : num_sms;
+  if (a.split3)
+    return launch_pdl(tc_gemm_kernel<GU_BN, GU_STAGES, EPI_SWIGLU_SPLIT3>, dim3(grid), dim3(NUM_THREADS),
+                      Cfg<GU_BN, GU_STAGES>::SMEM_BYTES, st, a.tm_x, a.tm_w, ep, m_blocks, n_blocks, 6 * k_blocks, k_blocks);
   return launch_pdl(tc_gemm_kernel<GU_BN, GU_STAGES, EPI_SWIGLU>, dim3(grid), dim3(NUM_THREADS),
-                    Cfg<GU_BN, GU_STAGES>::SMEM_BYTES, st, a.tm_x, a.tm_w, ep, m_blocks, n_blocks, k_blocks);
+                    Cfg<GU_BN, GU_STAGES>::SMEM_BYTES, st, a.tm_x, a.tm_w, ep, m_blocks, n_blocks, k_blocks, k_blocks);
 }
 
 cudaError_t launch_tc_down(const TcDownArgs& a, int num_sms, cudaStream_t st) {
@@ -207,7 +220,7 @@ cudaError_t launch_tc_down(const TcDownArgs& a, int num_sms, cudaStream_t st) {
   const int tiles = m_blocks * n_blocks;
   const int grid = tiles < num_sms ? tiles : num_sms;
   return launch_pdl(tc_gemm_kernel<DN_BN, DN_STAGES, EPI_OUT>, dim3(grid), dim3(NUM_THREADS), Cfg<DN_BN, DN_STAGES>::SMEM_BYTES,
-                    st, a.tm_h, a.tm_w, ep, m_blocks, n_blocks, k_blocks);
+                    st, a.tm_h, a.tm_w, ep, m_blocks, n_blocks, a.split3 ? 6 * k_blocks : k_blocks, k_blocks);
 }
 
 }  // namespace mlpmoe

@@ -59,6 +59,32 @@ def test_config3_fade_full_size(lib):
         lib.mlpmoe_destroy(h)
 
 
+def test_config3_structured_fade_full_size(lib):
+    """The neuron-structured variant at the Llama-shaped layer of configs[2]: the set of removed neurons is decided by
+    float64 scores that both sides must add up identically (14336 neurons x 8192 terms), so it is compared exactly."""
+    B, n = 32, 2048
+    d_b = synth.equal_partition(I, B)
+    bits = synth.layer_weights(3, 0, D, I, 0.02, bf16=True)
+    host = [synth.bf16_bits_to_f32(b) for b in bits]
+    dev = [dev_bf16(b) for b in bits]
+    h = lib.mlpmoe_create(D, I, d_b, dev[0], dev[1], dev[2], None, lib.MLPMOE_BF16, lib.MLPMOE_LAYOUT_PAPER, n, stream_ptr())
+    try:
+        lib.mlpmoe_fade_structured(h, None, stream_ptr())
+        Fg, Fu = oracle.fade_structured(host[0], host[1], d_b)
+        assert lib.mlpmoe_get_klist(h, B, I) == oracle.surviving_set([1.0] * B, Fg, Fu, host[2], d_b)
+        left = lib.mlpmoe_get_active_neurons(h)
+        assert left == I - sum((9 * b * 448) // (10 * B) for b in range(B))
+        xb = synth.f32_to_bf16_bits(synth.tokens(3, n, D))
+        y = torch.empty((n, D), dtype=torch.float32, device="cuda")
+        lib.mlpmoe_forward(h, dev_bf16(xb), y, n, stream_ptr())
+        torch.cuda.synchronize()
+        rows = [0, 255, 256, 1000, n - 1]
+        ref = oracle.mlpmoe_forward(synth.bf16_bits_to_f32(xb[rows]), Fg, Fu, host[2], d_b)
+        assert rel_err(y.cpu().numpy()[rows], ref) <= TOL_BF16
+    finally:
+        lib.mlpmoe_destroy(h)
+
+
 @pytest.fixture(scope="module")
 def llama_stack():
     """Seeded bf16 weights of the 32 Llama-shaped layers: bit patterns on the host, tensors on the device."""

@@ -125,6 +125,41 @@ def test_fade_masks_bit_exact(lib, bf16):
 
 
 @pytest.mark.parametrize("bf16", [True, False])
+def test_structured_fade_bit_exact_and_forward(lib, bf16):
+    """The neuron-structured Fade variant: removed neurons, schedule and forward against the oracle; composes
+    with pruning and with the paper's Fade; idempotent."""
+    d, I, d_b = 192, 640, [64, 192, 128, 256]
+    c = Case((107, int(bf16)), d, I, d_b, bf16=bf16, std=0.02, alpha=[1.0, 0.9, 1.1, 1.05])
+    for w in (c.bits, c.host) if bf16 else (c.host,):
+        w[0][:, 70] = w[0][:, 71]                    # equal scores: the lower index goes first
+        w[1][:, 70] = w[1][:, 71]
+    c.dev = [dev_bf16(b) for b in c.bits] if bf16 else [dev_f32(w) for w in c.host]
+    h = c.create(lib, 256)
+    try:
+        for s in (None, [0.0, 0.5, 0.3, 0.99]):
+            lib.mlpmoe_fade_structured(h, s, stream_ptr())
+        Fg, Fu = oracle.fade_structured(c.host[0], c.host[1], d_b)
+        Fg, Fu = oracle.fade_structured(Fg, Fu, d_b, [0.0, 0.5, 0.3, 0.99])
+        wg = torch.empty_like(c.dev[0]); wu = torch.empty_like(c.dev[1])
+        lib.mlpmoe_get_weights(h, wg, wu, None, stream_ptr())
+        torch.cuda.synchronize()
+        got = [synth.bf16_bits_to_f32(bits_of(w)) if bf16 else w.cpu().numpy() for w in (wg, wu)]
+        assert np.array_equal(got[0], Fg) and np.array_equal(got[1], Fu)
+        assert lib.mlpmoe_get_klist(h, 4, I) == oracle.surviving_set(c.alpha, Fg, Fu, c.host[2], d_b)
+        gone = I - lib.mlpmoe_get_active_neurons(h)
+        assert gone == int(np.sum(~np.any(Fg != 0, axis=0))) and gone > 200
+        for n in (150, 5):
+            xh, xd = c.tokens((107, n), n)
+            y = run_forward(lib, h, xd, n, d)
+            assert rel_err(y, oracle.mlpmoe_forward(xh, Fg, Fu, c.host[2], d_b, c.alpha)) <= (TOL_BF16 if bf16 else TOL_FP32)
+        with pytest.raises(lib.MlpmoeError) as e:
+            lib.mlpmoe_fade_structured(h, [0.0, 1.0, 0.1, 0.1], stream_ptr())
+        assert e.value.status == lib.MLPMOE_ERR_BAD_SCHEDULE
+    finally:
+        lib.mlpmoe_destroy(h)
+
+
+@pytest.mark.parametrize("bf16", [True, False])
 def test_prune_schedule_bit_exact_and_forward(lib, bf16):
     """Compensated Pruning (Section 3.3): effective gates, K-list and the forward."""
     d, I, B = 128, 640, 8

@@ -188,6 +188,53 @@ def test_planted_fade_mistakes_are_caught(monkeypatch):
     assert not top_k_ok()
 
 
+# ------------------------------------------------ structured variant -------- #
+def test_structured_fade_brute_force_and_counts():
+    """The neuron-structured variant against a scalar restatement: per branch, sort the neurons by
+    (score, index) with scores summed term by term in plain Python floats, drop the first floor(s d_b)."""
+    rng = np.random.default_rng(41)
+    d, d_b = 6, [4, 5, 7, 8]
+    I = sum(d_b)
+    Wg = rng.standard_normal((d, I)).astype(np.float32)
+    Wu = rng.standard_normal((d, I)).astype(np.float32)
+    Wg[:, 10] = Wg[:, 9]; Wu[:, 10] = Wu[:, 9]                     # a tie inside branch 2: the lower index goes first
+    s = [0, Fraction(2, 5), 0.5, Fraction(7, 8)]
+    Fg, Fu = oracle.fade_structured(Wg, Wu, d_b, s)
+    offs = oracle.branch_offsets(d_b)
+    for b in range(4):
+        scores = []
+        for j in range(offs[b], offs[b + 1]):
+            acc = 0.0
+            for k in range(d):
+                acc += float(Wg[k, j]) * float(Wg[k, j])
+            for k in range(d):
+                acc += float(Wu[k, j]) * float(Wu[k, j])
+            scores.append((acc, j))
+        q = int(math.floor(Fraction(s[b]) * d_b[b]))
+        assert q == oracle.fade_structured_count(s[b], d_b[b])
+        gone = {j for _, j in sorted(scores)[:q]}
+        for j in range(offs[b], offs[b + 1]):
+            if j in gone:
+                assert not Fg[:, j].any() and not Fu[:, j].any()
+            else:
+                assert np.array_equal(Fg[:, j], Wg[:, j]) and np.array_equal(Fu[:, j], Wu[:, j])
+    assert 9 in {j for j in range(I) if not Fg[:, j].any()} or 10 not in {j for j in range(I) if not Fg[:, j].any()}
+    # exact small integers: scores 2 k^2 for column k; the default schedule on B = 2 drops floor(0.45 * 4) = 1 of branch 1
+    Wi = np.tile(np.arange(1, 9, dtype=np.float32), (3, 1))
+    assert oracle.neuron_scores(Wi, Wi).tolist() == [6.0 * k * k for k in range(1, 9)]
+    Gi, Ui = oracle.fade_structured(Wi, Wi, [4, 4])
+    assert [j for j in range(8) if not Gi[:, j].any()] == [4]
+    # idempotent, inputs untouched, dead neurons leave the schedule
+    G2, U2 = oracle.fade_structured(Fg, Fu, d_b, s)
+    assert np.array_equal(G2, Fg) and np.array_equal(U2, Fu)
+    Wd = rng.standard_normal((I, d)).astype(np.float32)
+    _, segs = oracle.surviving_set([1.0] * 4, Fg, Fu, Wd, d_b)
+    assert sum(l for _, l in segs) == I - sum(oracle.fade_structured_count(s[b], d_b[b]) for b in range(4))
+    x = rng.standard_normal((3, d))
+    np.testing.assert_allclose(oracle.mlpmoe_forward(x, Fg, Fu, Wd, d_b), oracle.mlpmoe_forward_skiplist(x, Fg, Fu, Wd, d_b, [1.0] * 4),
+                               rtol=1e-12, atol=1e-12)
+
+
 # -------------------------------------------------------------- pruning ----- #
 def test_compensation_values():
     a = oracle.prune_alpha([1.0] * 16, oracle.first_k_keep(16, 12))
