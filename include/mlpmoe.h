@@ -131,6 +131,20 @@ mlpmoe_status_t mlpmoe_prune(mlpmoe_handle_t h, const uint8_t* keep, int32_t com
 /* The paper's literal rule (Section 3.3): keep branches b < K, alpha_b = sqrt(B/K). 1 <= K <= B. */
 mlpmoe_status_t mlpmoe_prune_first_k(mlpmoe_handle_t h, int32_t K, void* stream);
 
+/*
+ * Fast fp32 mode for an MLPMOE_FP32 layer: the layer equation of Section 3.1 on the tensor cores at
+ * fp32-grade accuracy.  Every fp32 operand v is held as three bf16 pieces p0 = bf16(v),
+ * p1 = bf16(v - p0), p2 = bf16(v - p0 - p1) (24 significand bits together); a product a * b is the sum
+ * of the six piece products a0 b0, a0 b1, a0 b2, a1 b0, a1 b1, a2 b0 (what is dropped is below
+ * 2^-23 of |a b|), accumulated in fp32.  Both GEMMs run this way (the K loop is six times as
+ * long), the intermediate activation is kept as the three-way split of its fp32 value, SiLU uses
+ * the accurate exponential.  Used by the forward calls for n_tokens > 64; fewer tokens keep the
+ * plain fp32 arithmetic.  Enabling allocates the split copies (1.5 x the fp32 weights, and
+ * activations for max_tokens) and is re-applied by later fade / prune calls; `enable` = 0 switches
+ * back.  MLPMOE_ERR_UNSUPPORTED for a bf16 layer.  Not in the paper: an implementation mode.
+ */
+mlpmoe_status_t mlpmoe_set_fast_fp32(mlpmoe_handle_t h, int32_t enable, void* stream);
+
 /* ------------------------------------------------------------------------- *
  * Forward (Section 3.1 layer equation).  Enqueues on `stream`, never
  * synchronises, allocates nothing.  (The first call above 128 tokens with a new

@@ -38,6 +38,7 @@ SIGNATURES = {
     "mlpmoe_destroy": (None, [c_void_p]),
     "mlpmoe_share_workspace": (c_int32, [c_void_p, c_void_p]),
     "mlpmoe_fade": (c_int32, [c_void_p, POINTER(c_double), c_void_p]),
+    "mlpmoe_set_fast_fp32": (c_int32, [c_void_p, c_int32, c_void_p]),
     "mlpmoe_fade_structured": (c_int32, [c_void_p, POINTER(c_double), c_void_p]),
     "mlpmoe_prune": (c_int32, [c_void_p, POINTER(c_uint8), c_int32, c_void_p]),
     "mlpmoe_prune_first_k": (c_int32, [c_void_p, c_int32, c_void_p]),
@@ -144,6 +145,10 @@ def mlpmoe_share_workspace(h: int, donor: int) -> None:
 
 def mlpmoe_fade(h: int, s: Optional[Sequence[float]] = None, stream=None) -> None:
     _check(lib.mlpmoe_fade(h, _arr(s, c_double), _stream(stream)), "mlpmoe_fade")
+
+
+def mlpmoe_set_fast_fp32(h: int, enable: bool = True, stream=None) -> None:
+    _check(lib.mlpmoe_set_fast_fp32(h, 1 if enable else 0, _stream(stream)), "mlpmoe_set_fast_fp32")
 
 
 def mlpmoe_fade_structured(h: int, s: Optional[Sequence[float]] = None, stream=None) -> None:

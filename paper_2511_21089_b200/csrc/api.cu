@@ -194,6 +194,11 @@ struct mlpmoe_layer_s {
   int plan_npad = 0;
   CUtensorMap plan_tm_x;                                    // normalised rows [n x d] as the kernels' token operand
   WaitCfg wait;                                             // bounded-wait limits of this handle's launches (test hook)
+  // fast fp32 mode (fp32 layers): three-way bf16 splits of the packed operands and of the activations
+  bool fast32 = false;
+  int64_t dp = 0;                                           // d rounded up to the 64-wide K-step
+  void *Wgu3 = nullptr, *WdT3 = nullptr;                    // [2 Ipad_max x 3 dp], [d x 3 Ipad_max] bf16
+  void *X3 = nullptr, *H3 = nullptr;                        // [max_tokens x 3 dp], [max_tokens x 3 Ipad_max] bf16
   uint32_t* counters = nullptr;
   uint32_t* block_done = nullptr;                           // [2 x ceil(max_tokens / 256)] gate|up completion counters
   int64_t max_blocks = 0;
@@ -240,8 +245,16 @@ void free_layer(mlpmoe_layer_s* h) {
   cudaFree(h->scale); cudaFree(h->src_row); cudaFree(h->row_nnz);
   cudaFree(h->fade_work); cudaFree(h->partial); cudaFree(h->counters); cudaFree(h->block_done); cudaFree(h->tile_sched); cudaFree(h->stack_dev); cudaFree(h->stack_counter); cudaFree(h->status);
   cudaFree(h->pstack_dev); cudaFree(h->pstack_items); cudaFree(h->pstack_counters); cudaFree(h->dec_tiled);
+  cudaFree(h->Wgu3); cudaFree(h->WdT3); cudaFree(h->X3); cudaFree(h->H3);
   ws_release(h->ws);
   delete h;
+}
+
+// Fast fp32 mode: the three-way bf16 splits of the current packed operands.
+mlpmoe_status_t refresh_fast32(mlpmoe_layer_s* h, cudaStream_t st) {
+  CK(launch_split3(static_cast<const float*>(h->Wgu), h->Wgu3, 2 * h->Ipad, h->d, h->dp, h->d, st));
+  CK(launch_split3(static_cast<const float*>(h->WdT), h->WdT3, h->d, h->Ipad, h->Ipad, h->Ipad, st));
+  return MLPMOE_OK;
 }
 
 // Recompute liveness, the K-list, the per-neuron scale and the packed operands from the
@@ -276,6 +289,10 @@ mlpmoe_status_t reschedule(mlpmoe_layer_s* h, cudaStream_t st) {
   CK(launch_gather_gateup(h->Wg_c, h->Wu_c, h->src_row, h->Wgu, n_active, h->Ipad, h->d, h->elem_size, st));
   CK(launch_gather_down_t(h->Wd_c, h->src_row, h->WdT, n_active, h->Ipad, h->d, h->elem_size, st));
   CK(cudaStreamSynchronize(st));    // the host vectors above go out of scope
+  if (h->fast32) {
+    mlpmoe_status_t fs = refresh_fast32(h, st);
+    if (fs != MLPMOE_OK) return fs;
+  }
   if (h->dtype == MLPMOE_BF16) {
     if (!make_tmap(&h->tm_wgu, h->Wgu, h->d, 2 * h->Ipad, h->d, 256)) return MLPMOE_ERR_CUDA;
     if (!make_tmap(&h->tm_wdt, h->WdT, h->Ipad, h->d, h->Ipad, 128)) return MLPMOE_ERR_CUDA;
@@ -312,6 +329,36 @@ mlpmoe_status_t forward_impl(mlpmoe_layer_s* h, const void* x, void* y, int64_t 
     return MLPMOE_ERR_INVALID_ARG;
   pdl_overlap_enabled() = !h->timing;
   if (y_dtype != MLPMOE_FP32 && !(y_dtype == MLPMOE_BF16 && h->dtype == MLPMOE_BF16)) return MLPMOE_ERR_UNSUPPORTED;
+  if (h->dtype == MLPMOE_FP32 && h->fast32 && n > kDecodeMaxTokens) {
+    // tensor-core path: every product of the two GEMMs as six bf16 piece products with fp32 accumulation
+    TcGateUpArgs g;
+    TcDownArgs dn;
+    CK(launch_split3(static_cast<const float*>(x), h->X3, n, h->d, h->dp, h->d, st));
+    if (!make_tmap(&g.tm_x, h->X3, 3 * h->dp, n, 3 * h->dp, 128)) return MLPMOE_ERR_CUDA;
+    if (!make_tmap(&g.tm_w, h->Wgu3, 3 * h->dp, 2 * h->Ipad, 3 * h->dp, 256)) return MLPMOE_ERR_CUDA;
+    g.scale = h->scale;
+    g.H = h->H3;
+    g.n = n; g.d = h->d; g.Ipad = h->Ipad;
+    g.status = h->status;
+    g.split3 = 1;
+    if (!make_tmap(&dn.tm_h, h->H3, 3 * h->Ipad, n, 3 * h->Ipad, 128)) return MLPMOE_ERR_CUDA;
+    if (!make_tmap(&dn.tm_w, h->WdT3, 3 * h->Ipad, h->d, 3 * h->Ipad, 128)) return MLPMOE_ERR_CUDA;
+    dn.R = residual;
+    dn.Y = y;
+    dn.y_bf16 = 0;
+    dn.n = n; dn.d = h->d; dn.Ipad = h->Ipad;
+    dn.status = h->status;
+    dn.split3 = 1;
+    const long e0 = rec_event(h, st);
+    CK(launch_tc_gateup(g, h->num_sms, st));
+    const long e1 = rec_event(h, st);
+    CK(launch_tc_down(dn, h->num_sms, st));
+    const long e2 = rec_event(h, st);
+    add_span(h, SPAN_GATEUP, e0, e1);
+    add_span(h, SPAN_DOWN, e1, e2);
+    h->launches += 3;
+    return MLPMOE_OK;
+  }
   if (h->dtype == MLPMOE_FP32) {
     float* H = static_cast<float*>(h->ws->H);
     const long e0 = rec_event(h, st);
@@ -785,6 +832,30 @@ mlpmoe_status_t mlpmoe_fade(mlpmoe_handle_t h, const double* s, void* stream) {
   CK(launch_fade(segs.data(), static_cast<int>(segs.size()), h->fade_work, h->elem_size, st));
   CK(cudaStreamSynchronize(st));     // segs is host memory read by an async copy
   return reschedule(h, st);
+}
+
+mlpmoe_status_t mlpmoe_set_fast_fp32(mlpmoe_handle_t h, int32_t enable, void* stream) {
+  if (!h) return MLPMOE_ERR_INVALID_ARG;
+  if (h->dtype != MLPMOE_FP32) return MLPMOE_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!enable) { h->fast32 = false; return MLPMOE_OK; }
+  if (h->Wgu3 == nullptr) {
+    h->dp = round_up(h->d, 64);
+    const size_t e2 = sizeof(__nv_bfloat16);
+    if (cudaMalloc(&h->Wgu3, static_cast<size_t>(2 * h->Ipad_max) * 3 * h->dp * e2) != cudaSuccess ||
+        cudaMalloc(&h->WdT3, static_cast<size_t>(h->d) * 3 * h->Ipad_max * e2) != cudaSuccess ||
+        cudaMalloc(&h->X3, static_cast<size_t>(h->max_tokens) * 3 * h->dp * e2) != cudaSuccess ||
+        cudaMalloc(&h->H3, static_cast<size_t>(h->max_tokens) * 3 * h->Ipad_max * e2) != cudaSuccess) {
+      cudaGetLastError();
+      cudaFree(h->Wgu3); cudaFree(h->WdT3); cudaFree(h->X3); cudaFree(h->H3);
+      h->Wgu3 = h->WdT3 = h->X3 = h->H3 = nullptr;
+      return MLPMOE_ERR_ALLOC;
+    }
+  }
+  mlpmoe_status_t rc = refresh_fast32(h, st);
+  if (rc != MLPMOE_OK) return rc;
+  h->fast32 = true;
+  return MLPMOE_OK;
 }
 
 mlpmoe_status_t mlpmoe_fade_structured(mlpmoe_handle_t h, const double* s, void* stream) {

@@ -69,7 +69,9 @@ __device__ __forceinline__ void epilogue_swiglu(uint32_t taddr, const EpiArgs& e
 
 // As epilogue_swiglu with the fp32 value h = silu(gate) * up * scale (accurate exp) written as its three-way
 // bf16 split: piece s of H[row, j] goes to column s * ep.cols + j of a row of 3 * ep.cols (= ep.ld) elements.
-__device__ __forceinline__ void epilogue_swiglu_split3(uint32_t taddr, const EpiArgs& ep, int64_t row, int64_t neuron0, int half) {
+// taddr2 != 0: a second accumulator of the same shape (the correction terms) is added to gate and up first.
+__device__ __forceinline__ void epilogue_swiglu_split3(uint32_t taddr, const EpiArgs& ep, int64_t row, int64_t neuron0, int half,
+                                                       uint32_t taddr2) {
   __nv_bfloat16* H = static_cast<__nv_bfloat16*>(ep.out);
 #pragma unroll 1
   for (int c = 0; c < half; c += 16) {
@@ -77,6 +79,17 @@ __device__ __forceinline__ void epilogue_swiglu_split3(uint32_t taddr, const Epi
     ptx::tmem_ld_32x16(taddr + c, g);
     ptx::tmem_ld_32x16(taddr + half + c, u);
     ptx::tmem_ld_wait();
+    if (taddr2 != 0) {
+      uint32_t g2[16], u2[16];
+      ptx::tmem_ld_32x16(taddr2 + c, g2);
+      ptx::tmem_ld_32x16(taddr2 + half + c, u2);
+      ptx::tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        g[i] = __float_as_uint(__uint_as_float(g[i]) + __uint_as_float(g2[i]));
+        u[i] = __float_as_uint(__uint_as_float(u[i]) + __uint_as_float(u2[i]));
+      }
+    }
     const int64_t col0 = neuron0 + c;
     uint32_t pk[3][8];
 #pragma unroll
@@ -109,12 +122,21 @@ __device__ __forceinline__ void epilogue_swiglu_split3(uint32_t taddr, const Epi
 }
 
 // Y[row, col_base + j] = (R[row, col_base + j] +) acc_j for j < bn, clipped to ep.cols (a multiple of 4).
-__device__ __forceinline__ void epilogue_out(uint32_t taddr, const EpiArgs& ep, int64_t row, int64_t col_base, int bn) {
+// taddr2 != 0: a second accumulator of the same shape is added first (fp32, round to nearest).
+__device__ __forceinline__ void epilogue_out(uint32_t taddr, const EpiArgs& ep, int64_t row, int64_t col_base, int bn,
+                                             uint32_t taddr2 = 0) {
 #pragma unroll 1
   for (int c = 0; c < bn; c += 32) {
     uint32_t a[32];
     ptx::tmem_ld_32x32(taddr + c, a);
     ptx::tmem_ld_wait();
+    if (taddr2 != 0) {
+      uint32_t b[32];
+      ptx::tmem_ld_32x32(taddr2 + c, b);
+      ptx::tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) a[i] = __float_as_uint(__uint_as_float(a[i]) + __uint_as_float(b[i]));
+    }
     const int64_t col0 = col_base + c;
     if (row < ep.rows) {
 #pragma unroll

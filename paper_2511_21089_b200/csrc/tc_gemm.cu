@@ -32,10 +32,14 @@ struct Cfg {
 template <int BN, int STAGES, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const EpiArgs ep,
-               int num_m_blocks, int num_n_blocks, int num_k_blocks, int kseg) {
+               int num_m_blocks, int num_n_blocks, int num_k_blocks, int kseg, int two_acc) {
   // K loop over num_k_blocks = terms * kseg blocks of 64: term t multiplies segment a_seg(t) of A's row by segment
   // b_seg(t) of B's row.  One term (kseg = num_k_blocks) is the plain product; the six terms of the fast fp32
   // mode pair the three-way splits of both operands as (0,0) (0,1) (0,2) (1,0) (1,1) (2,0).
+  // two_acc (six-term mode): the leading term (0,0) and the five correction terms, 2^-8 and less of it,
+  // accumulate in two accumulators that the epilogue adds.  The tensor cores' fp32 accumulation loses a
+  // little on every add in proportion to the running sum; keeping the number of adds into the large sum
+  // at a sixth, and the long tail of adds on a sum 2^-8 as large, keeps the total within fp32 round-off.
   using C = Cfg<BN, STAGES>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -47,6 +51,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  // accumulator buffers: two (the epilogue of a tile runs under the MMAs of the next) unless the two accumulators
+  // of a tile in two_acc mode already fill the 512 columns of tensor memory
+  const uint32_t acc_stride = two_acc ? 2u * BN : static_cast<uint32_t>(BN);
+  const int nbuf = 2u * acc_stride <= 512u ? 2 : 1;
+  const uint32_t tmem_cols = static_cast<uint32_t>(nbuf) * acc_stride;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -61,7 +70,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     fence_barrier_init();
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, C::TMEM_COLS);
+    tmem_alloc(tmem_slot, tmem_cols);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -109,8 +118,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         if (!mbar_wait_bounded(&tempty_bar[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+        const uint32_t d_main = tmem_base + static_cast<uint32_t>(acc) * acc_stride;
         for (int kb = 0; kb < num_k_blocks; ++kb) {
+          const bool corr = two_acc && kb >= kseg;               // a correction term
+          const uint32_t d_tmem = corr ? d_main + BN : d_main;
+          const int kb_first = corr ? kseg : 0;
           if (!mbar_wait_bounded(&full_bar[stage], phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * C::STAGE_BYTES);
@@ -119,15 +131,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing 16 elements along K inside the swizzled row = +32 bytes = +2 in the address field
-            umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb != kb_first || k != 0) ? 1u : 0u);
           }
           umma_commit(&empty_bar[stage]);       // stage is free once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         umma_commit(&tfull_bar[acc]);           // accumulator complete
-        acc ^= 1;
-        if (acc == 0) acc_phase ^= 1u;
+        if (++acc == nbuf) { acc = 0; acc_phase ^= 1u; }
       }
     }
   } else {
@@ -142,18 +153,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       if (!ok) break;
       tc_fence_after();
       const int64_t row = static_cast<int64_t>(m_blk) * BM + quad * 32 + lane;
-      const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * BN) + (static_cast<uint32_t>(quad * 32) << 16);
+      const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc) * acc_stride + (static_cast<uint32_t>(quad * 32) << 16);
       if (EPI == EPI_SWIGLU)
         epilogue_swiglu(taddr, ep, row, static_cast<int64_t>(n_blk) * (BN / 2), BN / 2);
       else if (EPI == EPI_SWIGLU_SPLIT3)
-        epilogue_swiglu_split3(taddr, ep, row, static_cast<int64_t>(n_blk) * (BN / 2), BN / 2);
+        epilogue_swiglu_split3(taddr, ep, row, static_cast<int64_t>(n_blk) * (BN / 2), BN / 2, two_acc ? taddr + BN : 0u);
       else
-        epilogue_out(taddr, ep, row, static_cast<int64_t>(n_blk) * BN, BN);
+        epilogue_out(taddr, ep, row, static_cast<int64_t>(n_blk) * BN, BN, two_acc ? taddr + BN : 0u);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tempty_bar[acc]);
-      acc ^= 1;
-      if (acc == 0) acc_phase ^= 1u;
+      if (++acc == nbuf) { acc = 0; acc_phase ^= 1u; }
     }
   }
 
@@ -162,7 +172,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, C::TMEM_COLS);
+    tmem_dealloc(tmem_base, tmem_cols);
   }
   if (threadIdx.x == 0 && *abort_flag) atomicExch(ep.status, kStatusTimeout);
 }
@@ -199,9 +209,9 @@ cudaError_t launch_tc_gateup(const TcGateUpArgs& a, int num_sms, cudaStream_t st
   const int grid = tiles < num_sms ? tiles : num_sms;
   if (a.split3)
     return launch_pdl(tc_gemm_kernel<GU_BN, GU_STAGES, EPI_SWIGLU_SPLIT3>, dim3(grid), dim3(NUM_THREADS),
-                      Cfg<GU_BN, GU_STAGES>::SMEM_BYTES, st, a.tm_x, a.tm_w, ep, m_blocks, n_blocks, 6 * k_blocks, k_blocks);
+                      Cfg<GU_BN, GU_STAGES>::SMEM_BYTES, st, a.tm_x, a.tm_w, ep, m_blocks, n_blocks, 6 * k_blocks, k_blocks, 1);
   return launch_pdl(tc_gemm_kernel<GU_BN, GU_STAGES, EPI_SWIGLU>, dim3(grid), dim3(NUM_THREADS),
-                    Cfg<GU_BN, GU_STAGES>::SMEM_BYTES, st, a.tm_x, a.tm_w, ep, m_blocks, n_blocks, k_blocks, k_blocks);
+                    Cfg<GU_BN, GU_STAGES>::SMEM_BYTES, st, a.tm_x, a.tm_w, ep, m_blocks, n_blocks, k_blocks, k_blocks, 0);
 }
 
 cudaError_t launch_tc_down(const TcDownArgs& a, int num_sms, cudaStream_t st) {
@@ -220,7 +230,7 @@ cudaError_t launch_tc_down(const TcDownArgs& a, int num_sms, cudaStream_t st) {
   const int tiles = m_blocks * n_blocks;
   const int grid = tiles < num_sms ? tiles : num_sms;
   return launch_pdl(tc_gemm_kernel<DN_BN, DN_STAGES, EPI_OUT>, dim3(grid), dim3(NUM_THREADS), Cfg<DN_BN, DN_STAGES>::SMEM_BYTES,
-                    st, a.tm_h, a.tm_w, ep, m_blocks, n_blocks, a.split3 ? 6 * k_blocks : k_blocks, k_blocks);
+                    st, a.tm_h, a.tm_w, ep, m_blocks, n_blocks, a.split3 ? 6 * k_blocks : k_blocks, k_blocks, a.split3 ? 1 : 0);
 }
 
 }  // namespace mlpmoe

@@ -39,6 +39,73 @@ def test_config1_fp32_equals_dense_swiglu(lib):
         lib.mlpmoe_destroy(h)
 
 
+def test_config1_fast_fp32_on_tensor_cores(lib):
+    """configs[0] in the fast fp32 mode (three-way bf16 split, six piece products per product, fp32 accumulation on the
+    tensor cores): same tolerance as the plain fp32 path, 1e-4 RMS, and the same result after the mode is switched off."""
+    c = Case((1, 0), 896, 4864, [608] * 8, bf16=False)
+    xh, xd = c.tokens((1, 0), 128)
+    h = c.create(lib, 128)
+    try:
+        ref = oracle.mlpmoe_forward(xh, *c.host, c.d_b)
+        y_plain = run_forward(lib, h, xd, 128, 896)
+        lib.mlpmoe_set_fast_fp32(h, True, stream_ptr())
+        launches = lib.mlpmoe_get_launch_count(h)
+        y_fast = run_forward(lib, h, xd, 128, 896)
+        assert lib.mlpmoe_get_launch_count(h) - launches == 3          # split, gate|up, down: the tensor-core path ran
+        e_plain, e_fast = rel_err(y_plain, ref), rel_err(y_fast, ref)
+        print(f"config 1: max|delta|/RMS plain fp32 {e_plain:.2e}, fast fp32 {e_fast:.2e}")
+        assert e_fast <= TOL_FP32
+        assert not np.array_equal(y_fast, y_plain)
+        lib.mlpmoe_set_fast_fp32(h, False, stream_ptr())
+        assert np.array_equal(run_forward(lib, h, xd, 128, 896), y_plain)
+    finally:
+        lib.mlpmoe_destroy(h)
+
+
+@pytest.mark.parametrize("d", [320, 328])
+@pytest.mark.parametrize("n", [65, 200, 391])
+def test_fast_fp32_ragged_with_fade_prune_and_stack(lib, d, n):
+    """Fast fp32 mode on ragged shapes (d_model = 328 pads the K segments), after Fade and pruning (the split copies
+    follow the schedule), with a residual, and as a two-layer stack."""
+    I, d_b = 400, [64, 160, 16, 160]
+    alpha = [1.0, 0.8, 1.2, -0.5]
+    c = Case((108, n, d), d, I, d_b, bf16=False, std=0.05, alpha=alpha)
+    xh, xd = c.tokens((108, n), n)
+    h = c.create(lib, 512)
+    try:
+        lib.mlpmoe_set_fast_fp32(h, True, stream_ptr())
+        ref = oracle.mlpmoe_forward(xh, *c.host, d_b, c.alpha)
+        assert rel_err(run_forward(lib, h, xd, n, d), ref) <= TOL_FP32
+        lib.mlpmoe_fade(h, None, stream_ptr())
+        keep = [True, True, False, True]
+        lib.mlpmoe_prune(h, keep, True, stream_ptr())
+        Fg, Fu = oracle.fade(c.host[0], c.host[1], d_b)
+        a = oracle.prune_alpha(c.alpha, keep)
+        ref = oracle.mlpmoe_forward(xh, Fg, Fu, c.host[2], d_b, a)
+        r = synth.normal_f32((108, n, 9), (n, d), 1.0)
+        y = dev_f32(r)
+        lib.mlpmoe_forward_ex(h, xd, y, n, y, lib.MLPMOE_FP32, stream_ptr())
+        torch.cuda.synchronize()
+        assert rel_err(y.cpu().numpy().astype(np.float64) - r, ref) <= TOL_FP32
+        xs = synth.normal_f32((108, 7, n), (n, d), 1.0)
+        xsd = dev_f32(xs)
+        lib.mlpmoe_stack_forward([h, h], xsd, n, 1e-6, stream_ptr())
+        torch.cuda.synchronize()
+        sref = oracle.stack_forward(xs, [(Fg, Fu, c.host[2], d_b, a)] * 2, bf16_activations=False)
+        assert rel_err(xsd.cpu().numpy(), sref) <= TOL_FP32
+        assert lib.mlpmoe_get_status(h) == lib.MLPMOE_OK
+    finally:
+        lib.mlpmoe_destroy(h)
+    cb = Case((108, 1), 128, 256, [128, 128], bf16=True, std=0.05)
+    hb = cb.create(lib, 64)
+    try:
+        with pytest.raises(lib.MlpmoeError) as e:
+            lib.mlpmoe_set_fast_fp32(hb, True, stream_ptr())
+        assert e.value.status == lib.MLPMOE_ERR_UNSUPPORTED
+    finally:
+        lib.mlpmoe_destroy(hb)
+
+
 @pytest.mark.parametrize("bf16", [True, False])
 @pytest.mark.parametrize("n", [65, 128, 200, 391])
 def test_small_layer_prefill(lib, bf16, n):
