@@ -334,6 +334,8 @@ class Bench:
             h = lib.mlpmoe_create(w["d"], w["I"], d_b, dev[0], dev[1], dev[2], alpha, lib.MLPMOE_BF16, lib.MLPMOE_LAYOUT_PAPER, w["n_max"], st)
             if w.get("fade"):
                 lib.mlpmoe_fade(h, None, st)
+            if w.get("structured"):
+                lib.mlpmoe_fade_structured(h, None, st)
             if keep is not None:
                 lib.mlpmoe_prune(h, keep, True, st)
             if layers:
@@ -495,6 +497,42 @@ class Bench:
             out["roofline"] = None
         return out
 
+    def measure_fp32(self):
+        """configs[0] (one Qwen-shaped fp32 layer, B = 8, all alpha 1): the plain fp32 FMA path against the fast fp32
+        mode (six bf16 piece products per product on the tensor cores), at the configuration's 128 tokens and at 4096."""
+        torch, lib, st = self.torch, self.lib, self.st
+        c = synth.CONFIGS[1]
+        d, I, B = c["d_model"], c["d_inter"], c["B"]
+        w = synth.layer_weights(1, 0, d, I, 0.02, bf16=False)
+        dev = [torch.from_numpy(np.ascontiguousarray(a)).cuda() for a in w]
+        n_max = 4096
+        h = lib.mlpmoe_create(d, I, synth.equal_partition(I, B), dev[0], dev[1], dev[2], None, lib.MLPMOE_FP32, lib.MLPMOE_LAYOUT_PAPER, n_max, st)
+        out = {"workload": f"configs[0]: single Qwen2.5-0.5B-shaped layer, fp32 weights and activations, B={B}, alpha=1"}
+        try:
+            for n in (c["n"], n_max):
+                x = torch.from_numpy(synth.tokens(1, n, d)).cuda()
+                y = torch.empty((n, d), dtype=torch.float32, device="cuda")
+                res = {}
+                for mode in ("plain", "fast"):
+                    lib.mlpmoe_set_fast_fp32(h, mode == "fast", st)
+                    for _ in range(5):
+                        lib.mlpmoe_forward(h, x, y, n, st)
+                    steps = 50
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    torch.cuda.synchronize()
+                    e0.record(self.stream)
+                    for _ in range(steps):
+                        lib.mlpmoe_forward(h, x, y, n, st)
+                    e1.record(self.stream)
+                    torch.cuda.synchronize()
+                    ms = e0.elapsed_time(e1) / steps
+                    res[mode] = {"ms_per_step": ms, "tokens_per_s": n / (ms * 1e-3), "tflops": 6.0 * n * d * I / (ms * 1e-3) / 1e12}
+                res["speedup_fast_over_plain"] = res["plain"]["ms_per_step"] / res["fast"]["ms_per_step"]
+                out[f"n{n}"] = res
+        finally:
+            lib.mlpmoe_destroy(h)
+        return out
+
     def is_one_launch(self, w):
         """Whether a stack call of workload w is one persistent launch (decode always; prefill when the layers stay in L2)."""
         if not w["stack"]:
@@ -536,7 +574,19 @@ def run_ours(args):
         hs = b.create_layers(wf)
         extras["c3_llama_layer_fade"] = b.measure(wf, hs, 300, 20)
         b.destroy(hs)
+        # the same layer under the neuron-structured Fade variant (same schedule, whole neurons removed): the only
+        # form of Fade that takes work off the dense tensor-core tiles
+        ws = dict(wf, fade=False, structured=True,
+                  label=wf["label"].replace("Fractal Fade s_b=0.9b/B", "neuron-structured Fade variant (labelled; not the paper's element-wise mask), s_b=0.9b/B"))
+        hs = b.create_layers(ws)
+        extras["c3_llama_layer_structured_fade"] = b.measure(ws, hs, 300, 20, e2e=False)
+        extras["c3_llama_layer_structured_fade"]["time_ratio_over_elementwise_fade"] = \
+            extras["c3_llama_layer_structured_fade"]["ms_per_step"] / extras["c3_llama_layer_fade"]["ms_per_step"]
+        extras["c3_llama_layer_structured_fade"]["neuron_ratio"] = \
+            extras["c3_llama_layer_structured_fade"]["surviving_neurons_per_layer"] / extras["c3_llama_layer_fade"]["surviving_neurons_per_layer"]
+        b.destroy(hs)
         b.drop_weights()
+        extras["c1_qwen_layer_fp32"] = b.measure_fp32()
         # configs[1]: the 24-layer Qwen-shaped stack
         wq = workload("qwen_stack")
         wq["n_max"] = wq["n"]
