@@ -103,7 +103,15 @@ def layer_inputs(layer: int, w, bits_cache=None):
 # workload, from the committed ncu summary under profiles/ named beside each figure; valid only while
 # the kernel's sources are the ones that were profiled (hash of the files), else reported as null.
 TRAFFIC = {
-    # workload name: (bytes per launch, source files, sha256[:16] of their concatenation, profile)
+    # workload key: (bytes per launch, source files, sha256[:16] of their concatenation, profile)
+    "llama_prefill": ((6234150144 + 627657728 + 5631617792 + 619579904) / 2, ('tc_layer.cu', 'tc_common.cuh', 'ptx.cuh'), "61d5a0e50491c749",
+                      "profiles/tc_layer_kernel_llama_c5_16384tokens.md (mean of the two layers captured at the headline shape)"),
+    "qwen_stack": (861574656 + 955400960, ('tc_stack.cu', 'tc_common.cuh', 'ptx.cuh'), "f920260a14cffc56", "profiles/tc_stack_kernel_qwen_c2_24layers.md"),
+    # decode: captured on 4 of the 32 layers; a launch streams its layers' weights once, so traffic scales with the layers
+    "llama_decode_1": ((1470823936 + 4195840) * 8, ('decode_fused.cu', 'ptx.cuh'), "41ae9186018dac22", "profiles/decode_fused_kernel_llama_c4_4layers.md"),
+    "llama_decode_8": ((1467553280 + 4698368) * 8, ('decode_fused.cu', 'ptx.cuh'), "41ae9186018dac22", "profiles/decode_fused_kernel_llama_c4_4layers.md"),
+    "llama_decode_32": ((1413513472 + 10400768) * 8, ('decode_stack.cu', 'ptx.cuh'), "925b810b9d6e3a09", "profiles/decode_stack_kernel_llama_c4_4layers.md"),
+    "llama_decode_64": ((1416810752 + 15351040) * 8, ('decode_stack.cu', 'ptx.cuh'), "925b810b9d6e3a09", "profiles/decode_stack_kernel_llama_c4_4layers.md"),
 }
 
 
@@ -115,11 +123,19 @@ def sources_sha(files) -> str:
     return h.hexdigest()[:16]
 
 
-def traffic_for(name: str):
+def traffic_for(w):
+    """DRAM bytes per launch of workload w's dominant kernel, if w is one of the captured shapes."""
+    name = None
+    if w["name"] == "llama_prefill" and (w["n"], w["B"], w["ratio"], w["L"]) == (HEADLINE["tokens"], HEADLINE["branches"], HEADLINE["ratio"], 32):
+        name = "llama_prefill"
+    elif w["name"] == "qwen_stack" and (w["n"], w["L"]) == (synth.CONFIGS[2]["n"], synth.CONFIGS[2]["layers"]):
+        name = "qwen_stack"
+    elif w["name"] == "llama_decode" and not w.get("prune_k") and w["L"] == 32:
+        name = f"llama_decode_{w['n']}"
     if name not in TRAFFIC:
         return None
     nbytes, files, sha, _ = TRAFFIC[name]
-    return nbytes if sources_sha(files) == sha else None
+    return float(nbytes) if sources_sha(files) == sha else None
 
 
 def peaks():
@@ -464,7 +480,7 @@ class Bench:
                 kernel = ("decode_fused_kernel" if n <= 13 else "decode_stack_kernel") + \
                     ": whole stack in one persistent launch (bulk-copy weight ring + tcgen05)"
                 out["roofline"] = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                                   "frac": achieved / pk["hbm_gbs"], "traffic": traffic_for(w["name"] + f"_{n}"),
+                                   "frac": achieved / pk["hbm_gbs"], "traffic": traffic_for(w),
                                    "peak_source": pk["source"] + " (copy bandwidth)", "avg_launch_us": main_ms * 1e3,
                                    "launches_timed": int(kcnt[0]), "share": share, "frac_of_nominal": achieved / 8000.0}
             elif n <= 64:
@@ -482,7 +498,7 @@ class Bench:
                           "tc_layer_kernel: gate|up GEMM + SiLU*up epilogue, then down GEMM + residual add (tcgen05, CTA pairs, one "
                           "launch per layer)")
                 rf = {"bound": "tensor", "kernel": kernel, "achieved": achieved, "unit": "TFLOP/s",
-                      "traffic": traffic_for(w["name"]), "avg_launch_us": main_ms * 1e3, "launches_timed": int(kcnt[0]), "share": share,
+                      "traffic": traffic_for(w), "avg_launch_us": main_ms * 1e3, "launches_timed": int(kcnt[0]), "share": share,
                       "frac_of_nominal": achieved / 2250.0}
                 rf.update(pick_frac(achieved, pk, region_s))
                 if kernel_mhz:
