@@ -560,6 +560,12 @@ def run_ours(args):
     b = Bench(args)
     lib = b.lib
     single = args.workload is not None
+    if args.workload == "qwen_layer_fp32":
+        # the fp32 block of the default line by itself (profiling captures of the fast fp32 kernels)
+        out = b.measure_fp32()
+        if b.rank == 0:
+            print(json.dumps({"configs": {"c1_qwen_layer_fp32": out}}))
+        return
     w = workload(args.workload or HEADLINE["name"], args.layers, args.tokens, args.branches, args.ratio, args.prune_k)
     w["n_max"] = w["n"]
     layers = b.create_layers(w)
@@ -646,7 +652,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--layers", type=int, default=None, help="fewer layers of the same stack (profiling captures only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=None, choices=["qwen_stack", "llama_decode", "llama_layer_fade", "llama_prefill"],
+    ap.add_argument("--workload", default=None, choices=["qwen_stack", "llama_decode", "llama_layer_fade", "llama_prefill", "qwen_layer_fp32"],
                     help="measure this workload alone (default: the headline workload plus the other configurations)")
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--branches", type=int, default=None)

@@ -8,6 +8,7 @@ from .mlpmoe_oracle import (  # noqa: F401
     silu,
     branch_forward,
     mlpmoe_forward,
+    routed_forward,
     fade_schedule,
     fade_position,
     fade_mask,

@@ -27,6 +27,10 @@ exact sqrt(B/K) values and the variance-preservation claim of Section 3.3.
 fade_structured / neuron_scores are a labelled variant of this build (no passage
 of the paper defines them): pinned by a scalar brute force, the closed-form
 count of removed neurons and exact small-integer cases.
+routed_forward is a labelled extension too (the paper names dynamic routing as
+future work only): pinned by its two special cases that the paper does define
+(all branches selected = the layer; one shared set = Compensated Pruning,
+Section 3.3), by a scalar brute force and by hand-computed values.
 The paper's perplexity and generation-time figures need trained checkpoints
 and an unpublished text mixture: parity unpinned for those (out of scope).
 """
@@ -241,6 +245,41 @@ def prune_alpha(alpha: Sequence[float], keep: Sequence[bool], compensate: bool =
         raise ValueError("the keep set is empty")
     c = math.sqrt(B / K) if compensate else 1.0
     return [float(alpha[b]) * c if keep[b] else 0.0 for b in range(B)]
+
+
+def routed_forward(x, W_gate, W_up, W_down, d_b: Sequence[int], alpha: Sequence[float], select,
+                   compensate: bool = True) -> np.ndarray:
+    """Per-token branch selection, a labelled extension (NOT defined by the paper:
+    Section 7, Limitation 2, and the outlook of Section 8 only name dynamic routing
+    over branches as future work).  The rule, stated here: token t evaluates the
+    branches S_t = {b : select[t, b] != 0 and alpha_b != 0} and nothing else,
+
+        y_t = c_t * sum_{b in S_t} branch_b(x_t),   c_t = sqrt(B' / |S_t|),
+
+    B' = number of branches with alpha_b != 0: Section 3.3's compensation with the
+    token's own K = |S_t|.  |S_t| = 0 gives y_t = 0; compensate=False gives c_t = 1.
+    With every available branch selected it is mlpmoe_forward; with one set S shared
+    by all tokens and all alpha_b != 0 it is the layer after prune_alpha(alpha, S).
+    The selection itself (a router) is an input: the paper defines none."""
+    x = np.asarray(x, dtype=np.float64)
+    sel = np.asarray(select)
+    B = len(d_b)
+    if sel.shape != (x.shape[0], B):
+        raise ValueError("select must be [n_tokens x B]")
+    offs = branch_offsets(d_b, np.asarray(W_gate).shape[1])
+    avail = [b for b in range(B) if float(alpha[b]) != 0.0]
+    chosen = np.zeros((x.shape[0], B), dtype=bool)
+    for b in avail:
+        chosen[:, b] = sel[:, b] != 0
+    acc = np.zeros((x.shape[0], np.asarray(W_down).shape[1]), dtype=np.float64)
+    for b in avail:                      # ascending b: every token's sum runs in the layer equation's order
+        rows = np.nonzero(chosen[:, b])[0]
+        if rows.size:
+            acc[rows] += branch_forward(x[rows], W_gate, W_up, W_down, offs[b], offs[b + 1], float(alpha[b]))
+    k = chosen.sum(axis=1)
+    c = np.zeros(x.shape[0], dtype=np.float64)
+    c[k > 0] = np.sqrt(len(avail) / k[k > 0]) if compensate else 1.0
+    return c[:, None] * acc
 
 
 # --------------------------------------------------------------------------- #
