@@ -171,6 +171,36 @@ mlpmoe_status_t mlpmoe_forward_ex(mlpmoe_handle_t h, const void* x, void* y, int
                                   const float* residual, mlpmoe_dtype_t y_dtype, void* stream);
 
 /*
+ * Per-token branch selection (dynamic routing over branches).  A LABELLED
+ * EXTENSION: Section 7 (Limitation 2) and the outlook of Section 8 name routing
+ * over the branches as future work and define no rule; the rule here is this
+ * library's own, built from Section 3.1's branches and Section 3.3's compensation:
+ *     S_t = { b : select[t, b] != 0 and alpha_b != 0 }          (alpha_b: the layer's current gates)
+ *     y_t = c_t * sum_{b in S_t} branch_b(x_t),   c_t = sqrt(B' / |S_t|),
+ * B' = number of branches with alpha_b != 0; |S_t| = 0 gives y_t = 0; compensate = 0
+ * gives c_t = 1.  With every available branch selected this is mlpmoe_forward; with
+ * one set shared by all tokens on an unpruned layer it is the layer after
+ * mlpmoe_prune(keep = that set).  How the selection is made (a router) is the
+ * caller's business.
+ *   x       device, [n_tokens x d_model], the layer's dtype, 16-byte aligned
+ *   y       device, [n_tokens x d_model] fp32, 16-byte aligned
+ *   select  device, [n_tokens x B] row-major bytes
+ * Only the selected (token, branch) pairs are computed: the tokens of a branch are
+ * gathered into one block, the branch runs on it as a layer of its own (the kernels
+ * of mlpmoe_forward, fp32 output), and the blocks are summed back per token in
+ * ascending b.  The first call, and the first after a Fade or a prune, builds one
+ * packed single-branch layer per available branch (allocates about the layer's
+ * packed weights once more, plus max_tokens x min(B, 8) fp32 output rows, and
+ * synchronises); EVERY call synchronises `stream` once, to read the per-branch
+ * token counts.  Pays for prefill-sized batches; for a handful of tokens the
+ * per-branch launches cost more than the skipped branches save.
+ * Errors: MLPMOE_ERR_INVALID_ARG (NULL, misaligned, n_tokens > max_tokens),
+ * MLPMOE_ERR_ALLOC, MLPMOE_ERR_CUDA.
+ */
+mlpmoe_status_t mlpmoe_forward_routed(mlpmoe_handle_t h, const void* x, float* y, int64_t n_tokens,
+                                      const uint8_t* select, int32_t compensate, void* stream);
+
+/*
  * mlpmoe_forward on HOST buffers: copies x to the device, runs the layer, copies y
  * back and synchronises `stream`.  x_host: layer dtype, y_host: fp32.  Pinned host
  * memory makes the copies asynchronous; pageable memory works too.

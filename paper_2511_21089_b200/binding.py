@@ -44,6 +44,7 @@ SIGNATURES = {
     "mlpmoe_prune_first_k": (c_int32, [c_void_p, c_int32, c_void_p]),
     "mlpmoe_forward": (c_int32, [c_void_p, c_void_p, c_void_p, c_int64, c_void_p]),
     "mlpmoe_forward_ex": (c_int32, [c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int32, c_void_p]),
+    "mlpmoe_forward_routed": (c_int32, [c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int32, c_void_p]),
     "mlpmoe_forward_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_int64, c_void_p]),
     "mlpmoe_rmsnorm": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_float, c_int32, c_void_p]),
     "mlpmoe_stack_prepare": (c_int32, [POINTER(c_void_p), c_int32, c_int64, c_void_p]),
@@ -170,6 +171,12 @@ def mlpmoe_forward(h: int, x, y, n_tokens: int, stream=None) -> None:
 
 def mlpmoe_forward_ex(h: int, x, y, n_tokens: int, residual=None, y_dtype: int = MLPMOE_FP32, stream=None) -> None:
     _check(lib.mlpmoe_forward_ex(h, _ptr(x), _ptr(y), n_tokens, _ptr(residual), y_dtype, _stream(stream)), "mlpmoe_forward_ex")
+
+
+def mlpmoe_forward_routed(h: int, x, y, n_tokens: int, select, compensate: bool = True, stream=None) -> None:
+    """select: device uint8 [n_tokens x B]."""
+    _check(lib.mlpmoe_forward_routed(h, _ptr(x), _ptr(y), n_tokens, _ptr(select), 1 if compensate else 0, _stream(stream)),
+           "mlpmoe_forward_routed")
 
 
 def mlpmoe_forward_host(h: int, x_host, y_host, n_tokens: int, stream=None) -> None:

@@ -17,7 +17,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OUT = os.path.join(PKG, "libmlpmoe_b200.so")
 OBJDIR = os.path.join(ROOT, "_build")
-SOURCES = ["api.cu", "pack.cu", "simt_gemm.cu", "tc_gemm.cu", "tc_layer.cu", "tc_stack.cu", "decode.cu", "decode_stack.cu", "decode_fused.cu", "static_scratch.cu"]
+SOURCES = ["api.cu", "pack.cu", "route.cu", "simt_gemm.cu", "tc_gemm.cu", "tc_layer.cu", "tc_stack.cu", "decode.cu", "decode_stack.cu", "decode_fused.cu", "static_scratch.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 

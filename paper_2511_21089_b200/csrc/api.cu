@@ -152,6 +152,20 @@ mlpmoe_status_t check_partition(int64_t d_inter, int B, const int64_t* d_b, int6
   return sum == d_inter ? MLPMOE_OK : MLPMOE_ERR_BAD_PARTITION;
 }
 
+// Per-token branch selection (mlpmoe_forward_routed): one single-branch layer per available branch, made
+// from the parent's canonical weights and current gates, and the buffers of the grouping step.
+struct Routed {
+  int64_t version = -1;                    // parent's schedule version the children were built for
+  std::vector<mlpmoe_layer_s*> child;      // [B]; nullptr where alpha_b = 0
+  int n_avail = 0;
+  uint8_t* avail = nullptr;                // device [B]
+  int32_t *pos = nullptr, *lists = nullptr, *counts = nullptr, *rowbase = nullptr;   // device: [max_tokens x B], [B x max_tokens], [B], [B]
+  float* coef = nullptr;                   // device [max_tokens]
+  void *Xe = nullptr, *Ye = nullptr;       // gathered rows of one branch; outputs of the branches of one pass
+  int64_t ye_rows = 0;
+  std::vector<int32_t> counts_host, rowbase_host;
+};
+
 }  // namespace
 
 struct mlpmoe_layer_s {
@@ -187,6 +201,7 @@ struct mlpmoe_layer_s {
   int pstack_bn = 0;
   int64_t version = 0;                                      // bumped by every reschedule
   int64_t uid = 0;                                          // process-wide, never reused (a freed handle's address can be)
+  Routed* routed = nullptr;                                 // built by the first mlpmoe_forward_routed
   // what the last mlpmoe_stack_prepare / first mlpmoe_stack_forward set up for a stack that starts with this layer
   std::vector<int64_t> plan_key;
   int plan_kind = 0;                                        // PLAN_*
@@ -237,8 +252,18 @@ void add_span(mlpmoe_layer_s* h, int kind, long a, long b) {
   if (a >= 0 && b >= 0) h->spans.push_back({kind, static_cast<size_t>(a), static_cast<size_t>(b)});
 }
 
+void free_layer(mlpmoe_layer_s* h);
+void free_routed(Routed* r) {
+  if (!r) return;
+  for (mlpmoe_layer_s* c : r->child) free_layer(c);
+  cudaFree(r->avail); cudaFree(r->pos); cudaFree(r->lists); cudaFree(r->counts); cudaFree(r->rowbase); cudaFree(r->coef);
+  cudaFree(r->Xe); cudaFree(r->Ye);
+  delete r;
+}
+
 void free_layer(mlpmoe_layer_s* h) {
   if (!h) return;
+  free_routed(h->routed);
   for (cudaEvent_t e : h->events) cudaEventDestroy(e);
   cudaFree(h->Wg_c); cudaFree(h->Wu_c); cudaFree(h->Wd_c);
   cudaFree(h->Wgu); cudaFree(h->WdT);
@@ -684,24 +709,21 @@ mlpmoe_status_t run_prefill_stack(const mlpmoe_handle_t* layers, int32_t n_layer
   return MLPMOE_OK;
 }
 
-}  // namespace
-
-extern "C" {
-
-mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_inter, int32_t B, const int64_t* d_b,
-                              const void* W_gate, const void* W_up, const void* W_down, const float* alpha,
-                              mlpmoe_dtype_t dtype, mlpmoe_layout_t layout, int64_t max_tokens, void* stream) {
+// Layer construction.  `layout` is one of the public layouts or kLayoutCanonical (all three matrices
+// neuron-major, [d_inter x d_model]: what the handle keeps); with `share` the layer uses that
+// workspace instead of allocating one (it must be large enough).
+constexpr int kLayoutCanonical = 2;
+mlpmoe_status_t create_impl(mlpmoe_handle_t* out, int64_t d_model, int64_t d_inter, int32_t B, const int64_t* d_b,
+                            const void* W_gate, const void* W_up, const void* W_down, const float* alpha, mlpmoe_dtype_t dtype,
+                            int layout, int64_t max_tokens, Workspace* share, cudaStream_t st) {
   if (!out) return MLPMOE_ERR_INVALID_ARG;
   *out = nullptr;
   if (d_model <= 0 || d_inter <= 0 || max_tokens <= 0 || !W_gate || !W_up || !W_down) return MLPMOE_ERR_INVALID_ARG;
   if (dtype != MLPMOE_BF16 && dtype != MLPMOE_FP32) return MLPMOE_ERR_INVALID_ARG;
-  if (layout != MLPMOE_LAYOUT_PAPER && layout != MLPMOE_LAYOUT_LINEAR) return MLPMOE_ERR_INVALID_ARG;
   mlpmoe_status_t ps = check_partition(d_inter, B, d_b, 16);
   if (ps != MLPMOE_OK) return ps;
   if (d_model % 8 != 0) return MLPMOE_ERR_UNSUPPORTED;
   if (d_inter > (int64_t(1) << 30) || d_model > (int64_t(1) << 30)) return MLPMOE_ERR_UNSUPPORTED;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-
   int dev = 0;
   CK(cudaGetDevice(&dev));
   cudaDeviceProp prop;
@@ -739,14 +761,24 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
   h->max_splits = h->num_sms / m_blocks + 1;
   h->max_blocks = (max_tokens + 255) / 256;
   h->sched_capacity = h->max_blocks * (h->Ipad_max / 128 + 4 * ((d_model + 63) / 64)) + h->num_sms / 2 + 2;
-  h->ws = new (std::nothrow) Workspace();
-  bool ok = h->ws != nullptr;
-  if (ok) {
-    h->ws->refs = 1;
-    h->ws->max_tokens = max_tokens;
-    h->ws->Ipad_max = h->Ipad_max;
-    h->ws->d = d_model;
-    h->ws->elem_size = h->elem_size;
+  bool ok = true;
+  if (share) {
+    if (share->elem_size != h->elem_size || share->max_tokens < max_tokens || share->Ipad_max < h->Ipad_max || share->d < d_model) {
+      delete h;
+      return MLPMOE_ERR_INVALID_ARG;
+    }
+    h->ws = share;
+    share->refs += 1;
+  } else {
+    h->ws = new (std::nothrow) Workspace();
+    ok = h->ws != nullptr;
+    if (ok) {
+      h->ws->refs = 1;
+      h->ws->max_tokens = max_tokens;
+      h->ws->Ipad_max = h->Ipad_max;
+      h->ws->d = d_model;
+      h->ws->elem_size = h->elem_size;
+    }
   }
   ok = ok && cudaMalloc(&h->Wg_c, mat) == cudaSuccess && cudaMalloc(&h->Wu_c, mat) == cudaSuccess &&
        cudaMalloc(&h->Wd_c, mat) == cudaSuccess &&
@@ -762,10 +794,11 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
        cudaMalloc(reinterpret_cast<void**>(&h->stack_counter), sizeof(uint32_t) * 3 * kMaxStackLayers) == cudaSuccess &&
        cudaMalloc(&h->block_done, sizeof(uint32_t) * 2 * h->max_blocks) == cudaSuccess &&
        cudaMalloc(&h->tile_sched, sizeof(int32_t) * h->sched_capacity) == cudaSuccess &&
-       cudaMalloc(&h->status, kStatusBytes) == cudaSuccess &&
-       cudaMalloc(&h->ws->H, static_cast<size_t>(max_tokens) * h->Ipad_max * es) == cudaSuccess &&
-       cudaMalloc(&h->ws->xnorm, static_cast<size_t>(max_tokens) * d_model * es) == cudaSuccess &&
-       cudaMalloc(reinterpret_cast<void**>(&h->ws->yres), static_cast<size_t>(max_tokens) * d_model * sizeof(float)) == cudaSuccess;
+       cudaMalloc(&h->status, kStatusBytes) == cudaSuccess;
+  if (ok && !share)
+    ok = cudaMalloc(&h->ws->H, static_cast<size_t>(max_tokens) * h->Ipad_max * es) == cudaSuccess &&
+         cudaMalloc(&h->ws->xnorm, static_cast<size_t>(max_tokens) * d_model * es) == cudaSuccess &&
+         cudaMalloc(reinterpret_cast<void**>(&h->ws->yres), static_cast<size_t>(max_tokens) * d_model * sizeof(float)) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     free_layer(h);
@@ -779,7 +812,11 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
     return fail(MLPMOE_ERR_CUDA);
   // canonical copies: one row of d contiguous weights per intermediate neuron, for all three matrices
   cudaError_t e;
-  if (layout == MLPMOE_LAYOUT_PAPER) {
+  if (layout == kLayoutCanonical) {
+    e = cudaMemcpyAsync(h->Wg_c, W_gate, mat, cudaMemcpyDeviceToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->Wu_c, W_up, mat, cudaMemcpyDeviceToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->Wd_c, W_down, mat, cudaMemcpyDeviceToDevice, st);
+  } else if (layout == MLPMOE_LAYOUT_PAPER) {
     e = launch_transpose(W_gate, h->Wg_c, d_model, d_inter, h->elem_size, st);
     if (e == cudaSuccess) e = launch_transpose(W_up, h->Wu_c, d_model, d_inter, h->elem_size, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(h->Wd_c, W_down, mat, cudaMemcpyDeviceToDevice, st);
@@ -793,6 +830,83 @@ mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_i
   if (rc != MLPMOE_OK) return fail(rc);
   *out = h;
   return MLPMOE_OK;
+}
+
+// The per-branch layers and buffers of mlpmoe_forward_routed, (re)built when the parent's weights or
+// gates have changed since.  Allocates and synchronises `st`.
+constexpr int64_t kRoutedPassBranches = 8;      // Ye holds max_tokens x min(B, this) rows; more selected rows take more passes
+mlpmoe_status_t ensure_routed(mlpmoe_layer_s* h, cudaStream_t st) {
+  if (h->routed && h->routed->version == h->version) return MLPMOE_OK;
+  CK(cudaStreamSynchronize(st));           // earlier routed calls may still use what is replaced below
+  if (!h->routed) {
+    Routed* r = new (std::nothrow) Routed();
+    if (!r) return MLPMOE_ERR_ALLOC;
+    h->routed = r;
+    r->child.assign(h->B, nullptr);
+    r->ye_rows = h->max_tokens * (h->B < kRoutedPassBranches ? h->B : kRoutedPassBranches);
+    const size_t row = static_cast<size_t>(h->d) * h->elem_size;
+    if (cudaMalloc(reinterpret_cast<void**>(&r->avail), h->B) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&r->pos), sizeof(int32_t) * h->max_tokens * h->B) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&r->lists), sizeof(int32_t) * h->max_tokens * h->B) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&r->counts), sizeof(int32_t) * h->B) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&r->rowbase), sizeof(int32_t) * h->B) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&r->coef), sizeof(float) * h->max_tokens) != cudaSuccess ||
+        cudaMalloc(&r->Xe, row * h->max_tokens) != cudaSuccess ||
+        cudaMalloc(&r->Ye, sizeof(float) * static_cast<size_t>(h->d) * r->ye_rows) != cudaSuccess) {
+      cudaGetLastError();
+      free_routed(r);
+      h->routed = nullptr;
+      return MLPMOE_ERR_ALLOC;
+    }
+  }
+  Routed* r = h->routed;
+  for (mlpmoe_layer_s*& c : r->child) { free_layer(c); c = nullptr; }
+  r->version = -1;
+  // widest branch first: its workspace serves all the others
+  std::vector<int> order;
+  for (int b = 0; b < h->B; ++b)
+    if (h->alpha_eff[b] != 0.0f) order.push_back(b);
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return h->d_b[a] > h->d_b[b]; });
+  r->n_avail = static_cast<int>(order.size());
+  Workspace* ws = nullptr;
+  const size_t row = static_cast<size_t>(h->d) * h->elem_size;
+  for (int b : order) {
+    const size_t off = static_cast<size_t>(h->offs[b]) * row;
+    const int64_t width = h->d_b[b];
+    const float alpha = h->alpha_eff[b];
+    mlpmoe_layer_s* c = nullptr;
+    mlpmoe_status_t rc = create_impl(&c, h->d, width, 1, &width, static_cast<const char*>(h->Wg_c) + off,
+                                     static_cast<const char*>(h->Wu_c) + off, static_cast<const char*>(h->Wd_c) + off, &alpha, h->dtype,
+                                     kLayoutCanonical, h->max_tokens, ws, st);
+    if (rc != MLPMOE_OK) return rc;
+    // the child only ever runs forward: its canonical copies are not needed once the operands are packed
+    CK(cudaStreamSynchronize(st));
+    cudaFree(c->Wg_c); cudaFree(c->Wu_c); cudaFree(c->Wd_c);
+    c->Wg_c = c->Wu_c = c->Wd_c = nullptr;
+    c->wait = h->wait;
+    r->child[b] = c;
+    if (!ws) ws = c->ws;
+  }
+  std::vector<uint8_t> avail(h->B, 0);
+  for (int b : order) avail[b] = 1;
+  CK(cudaMemcpyAsync(r->avail, avail.data(), h->B, cudaMemcpyHostToDevice, st));
+  CK(cudaStreamSynchronize(st));
+  r->counts_host.assign(h->B, 0);
+  r->rowbase_host.assign(h->B, 0);
+  r->version = h->version;
+  return MLPMOE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+mlpmoe_status_t mlpmoe_create(mlpmoe_handle_t* out, int64_t d_model, int64_t d_inter, int32_t B, const int64_t* d_b,
+                              const void* W_gate, const void* W_up, const void* W_down, const float* alpha,
+                              mlpmoe_dtype_t dtype, mlpmoe_layout_t layout, int64_t max_tokens, void* stream) {
+  if (layout != MLPMOE_LAYOUT_PAPER && layout != MLPMOE_LAYOUT_LINEAR) return MLPMOE_ERR_INVALID_ARG;
+  return create_impl(out, d_model, d_inter, B, d_b, W_gate, W_up, W_down, alpha, dtype, static_cast<int>(layout), max_tokens, nullptr,
+                     static_cast<cudaStream_t>(stream));
 }
 
 void mlpmoe_destroy(mlpmoe_handle_t h) { free_layer(h); }
@@ -931,6 +1045,58 @@ mlpmoe_status_t mlpmoe_forward_ex(mlpmoe_handle_t h, const void* x, void* y, int
   return forward_impl(h, x, y, n_tokens, residual, y_dtype, static_cast<cudaStream_t>(stream));
 }
 
+mlpmoe_status_t mlpmoe_forward_routed(mlpmoe_handle_t h, const void* x, float* y, int64_t n, const uint8_t* select,
+                                      int32_t compensate, void* stream) {
+  if (!h || n < 0) return MLPMOE_ERR_INVALID_ARG;
+  if (n == 0) return MLPMOE_OK;
+  if (!x || !y || !select || n > h->max_tokens || !aligned16(x) || !aligned16(y)) return MLPMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  mlpmoe_status_t rc = ensure_routed(h, st);
+  if (rc != MLPMOE_OK) return rc;
+  Routed* r = h->routed;
+  const int B = h->B;
+  // group the tokens by branch; the per-branch counts come back to the host (one synchronisation per call)
+  CK(launch_route_scan(select, r->avail, n, B, h->max_tokens, r->pos, r->lists, r->counts, st));
+  CK(launch_route_coef(r->pos, n, B, r->n_avail, compensate ? 1 : 0, r->coef, st));
+  CK(cudaMemcpyAsync(r->counts_host.data(), r->counts, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  // passes: consecutive branches whose rows fit the output buffer together
+  std::vector<int> pass_end;               // one past the last branch of each pass
+  int64_t used = 0;
+  for (int b = 0; b < B; ++b) {
+    const int64_t cnt = r->counts_host[b];
+    if (used + cnt > r->ye_rows) {
+      pass_end.push_back(b);
+      used = 0;
+    }
+    r->rowbase_host[b] = static_cast<int32_t>(used);
+    used += cnt;
+  }
+  pass_end.push_back(B);
+  CK(cudaMemcpyAsync(r->rowbase, r->rowbase_host.data(), sizeof(int32_t) * B, cudaMemcpyHostToDevice, st));
+  const size_t row = static_cast<size_t>(h->d) * h->elem_size;
+  const size_t ye_row = sizeof(float) * static_cast<size_t>(h->d);     // branch outputs stay fp32 until they are summed
+  int b0 = 0;
+  for (size_t p = 0; p < pass_end.size(); ++p) {
+    for (int b = b0; b < pass_end[p]; ++b) {
+      const int64_t cnt = r->counts_host[b];
+      if (cnt == 0 || !r->child[b]) continue;
+      CK(launch_gather_rows(x, r->lists + static_cast<int64_t>(b) * h->max_tokens, cnt, row, r->Xe, st));
+      r->child[b]->timing = false;
+      rc = forward_impl(r->child[b], r->Xe, static_cast<char*>(r->Ye) + static_cast<size_t>(r->rowbase_host[b]) * ye_row, cnt, nullptr,
+                        MLPMOE_FP32, st);
+      if (rc != MLPMOE_OK) return rc;
+      h->launches += 1 + r->child[b]->launches;
+      r->child[b]->launches = 0;
+    }
+    CK(launch_route_combine(r->Ye, 0, r->pos, r->rowbase, r->coef, n, B, b0, pass_end[p], h->d, p == 0, y, st));
+    h->launches += 1;
+    b0 = pass_end[p];
+  }
+  h->launches += 2;
+  return MLPMOE_OK;
+}
+
 mlpmoe_status_t mlpmoe_forward_host(mlpmoe_handle_t h, const void* x_host, float* y_host, int64_t n, void* stream) {
   if (!h || n < 0) return MLPMOE_ERR_INVALID_ARG;
   if (n == 0) return MLPMOE_OK;
@@ -1058,7 +1224,12 @@ mlpmoe_status_t mlpmoe_get_status(mlpmoe_handle_t h) {
   uint32_t w = 0;
   CK(cudaDeviceSynchronize());
   CK(cudaMemcpy(&w, h->status, sizeof(w), cudaMemcpyDeviceToHost));
-  if (w == kStatusOk) return MLPMOE_OK;
+  // the per-branch layers of routed calls report through their parent
+  bool child_timeout = false;
+  if (h->routed)
+    for (mlpmoe_layer_s* c : h->routed->child)
+      if (c && mlpmoe_get_status(c) == MLPMOE_ERR_DEVICE_TIMEOUT) child_timeout = true;
+  if (w == kStatusOk) return child_timeout ? MLPMOE_ERR_DEVICE_TIMEOUT : MLPMOE_OK;
   // A kernel gave up: the dependency counters that its work items leave at zero in a normal run may hold
   // anything.  Re-arm the handle (the counters that are not zeroed before every launch, and the status word).
   CK(cudaMemset(h->block_done, 0, sizeof(uint32_t) * 2 * h->max_blocks));

@@ -76,6 +76,15 @@ cudaError_t launch_split3(const float* src, void* dst, int64_t rows, int64_t K, 
 cudaError_t launch_neuron_scores(const void* Wg_c, const void* Wu_c, double* score, int64_t I, int64_t d, int elem_size, cudaStream_t st);
 cudaError_t launch_zero_rows(void* A, void* B, const int32_t* rows_dev, int64_t n_rows, int64_t d, int elem_size, cudaStream_t st);
 
+// Per-token branch selection (route.cu): stable grouping of the tokens by selected branch, the per-token
+// compensation factor, the row gather, and the sum of the branches' output rows back into y.
+cudaError_t launch_route_scan(const uint8_t* select, const uint8_t* avail, int64_t n, int B, int64_t list_stride, int32_t* pos,
+                              int32_t* lists, int32_t* counts, cudaStream_t st);
+cudaError_t launch_route_coef(const int32_t* pos, int64_t n, int B, int n_avail, int compensate, float* coef, cudaStream_t st);
+cudaError_t launch_gather_rows(const void* src, const int32_t* list, int64_t n_rows, int64_t row_bytes, void* out, cudaStream_t st);
+cudaError_t launch_route_combine(const void* Ye, int ye_bf16, const int32_t* pos, const int32_t* rowbase, const float* coef, int64_t n,
+                                 int B, int b_lo, int b_hi, int64_t d, int first, float* y, cudaStream_t st);
+
 // Fade: exact rank selection on magnitude bit patterns, then masking (Section 3.2).
 struct FadeSeg {
   void* base;      // first element of the slice (contiguous m elements)

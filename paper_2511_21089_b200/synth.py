@@ -21,7 +21,7 @@ import numpy as np
 BASE_SEED = 20251121
 
 # tensor ids
-T_GATE, T_UP, T_DOWN, T_X, T_ALPHA, T_KEEP, T_PARTITION = range(7)
+T_GATE, T_UP, T_DOWN, T_X, T_ALPHA, T_KEEP, T_PARTITION, T_ROUTE = range(8)
 
 _BLOCK = 1 << 20
 
@@ -97,6 +97,18 @@ def keep_set(key: Sequence[int], B: int, n_drop: int) -> List[bool]:
     if n_drop:
         keep[_rng(key).choice(B, size=n_drop, replace=False)] = False
     return [bool(k) for k in keep]
+
+
+def route_select(key: Sequence[int], n: int, B: int, k: int) -> np.ndarray:
+    """Selection bytes [n, B] of a per-token routing: every token selects exactly k distinct
+    branches, uniformly by seed (the k smallest of B independent uniform draws)."""
+    if not (0 <= k <= B):
+        raise ValueError("k must lie in 0..B")
+    sel = np.zeros((n, B), dtype=np.uint8)
+    if k:
+        order = np.argsort(_rng(key).random((n, B)), axis=1, kind="stable")[:, :k]
+        np.put_along_axis(sel, order, 1, axis=1)
+    return sel
 
 
 def n_drop_for_ratio(B: int, ratio: float) -> int:
