@@ -549,6 +549,53 @@ class Bench:
             lib.mlpmoe_destroy(h)
         return out
 
+    def measure_routed(self, k=8):
+        """configs[2]'s Llama-shaped layer (B = 32 equal slices, no Fade) under per-token branch selection, every token
+        choosing k of the 32 branches uniformly by seed (a labelled extension: the paper names routing as future work
+        only), against the plain forward of the same layer on the same tokens."""
+        torch, lib, st = self.torch, self.lib, self.st
+        w = workload("llama_layer_fade")
+        w = dict(w, fade=False, n_max=w["n"])
+        n, d, B = w["n"], w["d"], w["B"]
+        hs = self.create_layers(w)
+        h = hs[0]
+        out = {"workload": f"configs[2] shapes: single Llama-3-8B-shaped layer, bf16, B={B} equal slices, {n} tokens, every token "
+                           f"selects {k} of {B} branches (seeded), compensation sqrt(B/k)"}
+        try:
+            xb = synth.f32_to_bf16_bits(rank_batch(w["cfg"], n, d, self.rank))
+            x = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).cuda()
+            y = torch.empty((n, d), dtype=torch.float32, device="cuda")
+            sel = torch.from_numpy(synth.route_select((synth.BASE_SEED, w["cfg"], synth.T_ROUTE), n, B, k)).cuda()
+            res = {}
+            for mode in ("dense", "routed"):
+                def step():
+                    if mode == "dense":
+                        lib.mlpmoe_forward(h, x, y, n, st)
+                    else:
+                        lib.mlpmoe_forward_routed(h, x, y, n, sel, True, st)
+                for _ in range(5):
+                    step()
+                steps = 50
+                l0 = lib.mlpmoe_get_launch_count(h)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                e0.record(self.stream)
+                for _ in range(steps):
+                    step()
+                e1.record(self.stream)
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1) / steps
+                frac = 1.0 if mode == "dense" else k / B
+                res[mode] = {"ms_per_step": ms, "tokens_per_s": n / (ms * 1e-3), "tflops": 6.0 * n * d * w["I"] * frac / (ms * 1e-3) / 1e12,
+                             "gpu_launches_per_step": (lib.mlpmoe_get_launch_count(h) - l0) / steps}
+            assert lib.mlpmoe_get_status(h) == lib.MLPMOE_OK
+            res["flop_ratio_routed_over_dense"] = k / B
+            res["time_ratio_routed_over_dense"] = res["routed"]["ms_per_step"] / res["dense"]["ms_per_step"]
+            out.update(res)
+        finally:
+            self.destroy(hs)
+        return out
+
     def is_one_launch(self, w):
         """Whether a stack call of workload w is one persistent launch (decode always; prefill when the layers stay in L2)."""
         if not w["stack"]:
@@ -560,6 +607,11 @@ def run_ours(args):
     b = Bench(args)
     lib = b.lib
     single = args.workload is not None
+    if args.workload == "llama_layer_routed":
+        out = b.measure_routed()
+        if b.rank == 0:
+            print(json.dumps({"configs": {"c3_llama_layer_routed": out}}))
+        return
     if args.workload == "qwen_layer_fp32":
         # the fp32 block of the default line by itself (profiling captures of the fast fp32 kernels)
         out = b.measure_fp32()
@@ -607,6 +659,7 @@ def run_ours(args):
         extras["c3_llama_layer_structured_fade"]["neuron_ratio"] = \
             extras["c3_llama_layer_structured_fade"]["surviving_neurons_per_layer"] / extras["c3_llama_layer_fade"]["surviving_neurons_per_layer"]
         b.destroy(hs)
+        extras["c3_llama_layer_routed"] = b.measure_routed()
         b.drop_weights()
         extras["c1_qwen_layer_fp32"] = b.measure_fp32()
         # configs[1]: the 24-layer Qwen-shaped stack
@@ -652,7 +705,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--layers", type=int, default=None, help="fewer layers of the same stack (profiling captures only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=None, choices=["qwen_stack", "llama_decode", "llama_layer_fade", "llama_prefill", "qwen_layer_fp32"],
+    ap.add_argument("--workload", default=None, choices=["qwen_stack", "llama_decode", "llama_layer_fade", "llama_prefill", "qwen_layer_fp32", "llama_layer_routed"],
                     help="measure this workload alone (default: the headline workload plus the other configurations)")
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--branches", type=int, default=None)

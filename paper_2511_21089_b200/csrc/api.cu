@@ -162,8 +162,20 @@ struct Routed {
   int32_t *pos = nullptr, *lists = nullptr, *counts = nullptr, *rowbase = nullptr;   // device: [max_tokens x B], [B x max_tokens], [B], [B]
   float* coef = nullptr;                   // device [max_tokens]
   void *Xe = nullptr, *Ye = nullptr;       // gathered rows of one branch; outputs of the branches of one pass
-  int64_t ye_rows = 0;
+  int64_t ye_rows = 0;                     // rows of Ye (and, grouped, of Xe and Hg)
   std::vector<int32_t> counts_host, rowbase_host;
+  // bf16 layers: all branches of a pass in ONE launch of the stack kernel, the branches as its "layers"
+  bool grouped = false;
+  TcStackLayer* recs = nullptr;            // device [B]
+  void* Hg = nullptr;                      // [ye_rows x h_pitch] bf16
+  int64_t h_pitch = 0;
+  int bn = 256;
+  int32_t* items = nullptr;                // device: work items + offsets of the current launch
+  int64_t items_cap = 0;
+  uint32_t* group_counters = nullptr;      // device [3 x B x blocks]
+  int64_t counters_cap = 0;
+  std::vector<int32_t> items_host, block_layer;
+  std::vector<int64_t> ipad_host;
 };
 
 }  // namespace
@@ -257,7 +269,7 @@ void free_routed(Routed* r) {
   if (!r) return;
   for (mlpmoe_layer_s* c : r->child) free_layer(c);
   cudaFree(r->avail); cudaFree(r->pos); cudaFree(r->lists); cudaFree(r->counts); cudaFree(r->rowbase); cudaFree(r->coef);
-  cudaFree(r->Xe); cudaFree(r->Ye);
+  cudaFree(r->Xe); cudaFree(r->Ye); cudaFree(r->recs); cudaFree(r->Hg); cudaFree(r->items); cudaFree(r->group_counters);
   delete r;
 }
 
@@ -843,7 +855,9 @@ mlpmoe_status_t ensure_routed(mlpmoe_layer_s* h, cudaStream_t st) {
     if (!r) return MLPMOE_ERR_ALLOC;
     h->routed = r;
     r->child.assign(h->B, nullptr);
+    r->grouped = h->dtype == MLPMOE_BF16 && h->B <= kMaxStackLayers;
     r->ye_rows = h->max_tokens * (h->B < kRoutedPassBranches ? h->B : kRoutedPassBranches);
+    if (r->grouped) r->ye_rows = round_up(r->ye_rows, 256) + 256 * static_cast<int64_t>(h->B);   // every branch's rows start a 256-row block
     const size_t row = static_cast<size_t>(h->d) * h->elem_size;
     if (cudaMalloc(reinterpret_cast<void**>(&r->avail), h->B) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&r->pos), sizeof(int32_t) * h->max_tokens * h->B) != cudaSuccess ||
@@ -851,7 +865,8 @@ mlpmoe_status_t ensure_routed(mlpmoe_layer_s* h, cudaStream_t st) {
         cudaMalloc(reinterpret_cast<void**>(&r->counts), sizeof(int32_t) * h->B) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&r->rowbase), sizeof(int32_t) * h->B) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&r->coef), sizeof(float) * h->max_tokens) != cudaSuccess ||
-        cudaMalloc(&r->Xe, row * h->max_tokens) != cudaSuccess ||
+        cudaMalloc(&r->Xe, row * (r->grouped ? r->ye_rows : h->max_tokens)) != cudaSuccess ||
+        (r->grouped && cudaMalloc(reinterpret_cast<void**>(&r->recs), sizeof(TcStackLayer) * h->B) != cudaSuccess) ||
         cudaMalloc(&r->Ye, sizeof(float) * static_cast<size_t>(h->d) * r->ye_rows) != cudaSuccess) {
       cudaGetLastError();
       free_routed(r);
@@ -886,6 +901,39 @@ mlpmoe_status_t ensure_routed(mlpmoe_layer_s* h, cudaStream_t st) {
     c->wait = h->wait;
     r->child[b] = c;
     if (!ws) ws = c->ws;
+  }
+  if (r->grouped) {
+    // one "layer" record per branch: its packed weights, and its columns of the shared H buffer
+    int64_t pitch = kGroup;
+    for (int b : order) pitch = std::max(pitch, r->child[b]->Ipad);
+    if (pitch > r->h_pitch) {
+      cudaFree(r->Hg);
+      r->Hg = nullptr;
+      r->h_pitch = 0;
+      if (cudaMalloc(&r->Hg, sizeof(__nv_bfloat16) * static_cast<size_t>(r->ye_rows) * pitch) != cudaSuccess) {
+        cudaGetLastError();
+        return MLPMOE_ERR_ALLOC;
+      }
+      r->h_pitch = pitch;
+    }
+    r->bn = tc_layer_down_bn(r->ye_rows, h->d, h->num_sms);
+    std::vector<TcStackLayer> recs(static_cast<size_t>(h->B));
+    std::memset(recs.data(), 0, sizeof(TcStackLayer) * recs.size());
+    r->ipad_host.assign(h->B, kGroup);
+    for (int b : order) {
+      mlpmoe_layer_s* c = r->child[b];
+      recs[b].tm_wgu = c->tm_wgu_pair;
+      if (!make_tmap(&recs[b].tm_h_st, r->Hg, c->Ipad, r->ye_rows, r->h_pitch, 32)) return MLPMOE_ERR_CUDA;
+      if (!make_tmap(&recs[b].tm_h_ld, r->Hg, c->Ipad, r->ye_rows, r->h_pitch, 128)) return MLPMOE_ERR_CUDA;
+      if (!make_tmap(&recs[b].tm_wdt, c->WdT, c->Ipad, h->d, c->Ipad, r->bn / 2)) return MLPMOE_ERR_CUDA;
+      recs[b].scale = c->scale;
+      recs[b].n1 = static_cast<int32_t>(c->Ipad / 128);
+      recs[b].kb2 = static_cast<int32_t>(c->Ipad / 64);
+      recs[b].ksplit = 1;
+      r->ipad_host[b] = c->Ipad;
+    }
+    CK(cudaMemcpyAsync(r->recs, recs.data(), sizeof(TcStackLayer) * recs.size(), cudaMemcpyHostToDevice, st));
+    CK(cudaStreamSynchronize(st));
   }
   std::vector<uint8_t> avail(h->B, 0);
   for (int b : order) avail[b] = 1;
@@ -1064,7 +1112,7 @@ mlpmoe_status_t mlpmoe_forward_routed(mlpmoe_handle_t h, const void* x, float* y
   std::vector<int> pass_end;               // one past the last branch of each pass
   int64_t used = 0;
   for (int b = 0; b < B; ++b) {
-    const int64_t cnt = r->counts_host[b];
+    const int64_t cnt = r->grouped ? round_up(r->counts_host[b], 256) : r->counts_host[b];
     if (used + cnt > r->ye_rows) {
       pass_end.push_back(b);
       used = 0;
@@ -1077,6 +1125,82 @@ mlpmoe_status_t mlpmoe_forward_routed(mlpmoe_handle_t h, const void* x, float* y
   const size_t row = static_cast<size_t>(h->d) * h->elem_size;
   const size_t ye_row = sizeof(float) * static_cast<size_t>(h->d);     // branch outputs stay fp32 until they are summed
   int b0 = 0;
+  for (size_t p = 0; r->grouped && p < pass_end.size(); ++p) {
+    // the pass's branches in one launch: gathered rows of branch b at rows rowbase[b] .. of Xe, 256-row blocks
+    r->block_layer.clear();
+    {
+      // about 8 blocks of 256 threads per SM over the pass's branches
+      int per_branch = (8 * h->num_sms + (pass_end[p] - b0) - 1) / (pass_end[p] - b0);
+      CK(launch_gather_branches(x, r->lists, h->max_tokens, r->counts, r->rowbase, b0, pass_end[p], row, r->Xe, per_branch, st));
+      h->launches += 1;
+    }
+    for (int b = b0; b < pass_end[p]; ++b) {
+      const int64_t cnt = r->counts_host[b];
+      if (cnt == 0 || !r->child[b]) continue;
+      // blocks are numbered by their position in Xe: the block index is the row offset / 256
+      const int first_block = r->rowbase_host[b] / 256, n_blk = static_cast<int>((cnt + 255) / 256);
+      if (static_cast<int>(r->block_layer.size()) < first_block + n_blk) r->block_layer.resize(first_block + n_blk, -1);
+      for (int q = 0; q < n_blk; ++q) r->block_layer[first_block + q] = b;
+    }
+    const int n_blocks = static_cast<int>(r->block_layer.size());
+    if (n_blocks > 0) {
+      // every block of a pass is in use (the branches' padded row ranges are laid end to end)
+      for (int q = 0; q < n_blocks; ++q)
+        if (r->block_layer[q] < 0) return MLPMOE_ERR_CUDA;
+      std::vector<int32_t> offs;
+      tc_stack_group_schedule(r->block_layer.data(), n_blocks, h->d, r->ipad_host.data(), r->bn, h->num_sms, &r->items_host, &offs);
+      const int64_t n_items = static_cast<int64_t>(r->items_host.size());
+      r->items_host.insert(r->items_host.end(), offs.begin(), offs.end());
+      const int64_t need_items = static_cast<int64_t>(r->items_host.size());
+      const int64_t need_counters = 3 * static_cast<int64_t>(B) * n_blocks;
+      if (need_items > r->items_cap || need_counters > r->counters_cap) {
+        CK(cudaStreamSynchronize(st));
+        cudaFree(r->items); cudaFree(r->group_counters);
+        r->items = nullptr; r->group_counters = nullptr;
+        r->items_cap = r->counters_cap = 0;
+        if (cudaMalloc(reinterpret_cast<void**>(&r->items), sizeof(int32_t) * 2 * need_items) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void**>(&r->group_counters), sizeof(uint32_t) * 2 * need_counters) != cudaSuccess) {
+          cudaGetLastError();
+          return MLPMOE_ERR_ALLOC;
+        }
+        r->items_cap = 2 * need_items;
+        r->counters_cap = 2 * need_counters;
+      }
+      CK(cudaMemcpyAsync(r->items, r->items_host.data(), sizeof(int32_t) * need_items, cudaMemcpyHostToDevice, st));
+      if (p + 1 < pass_end.size()) CK(cudaStreamSynchronize(st));     // items_host is rebuilt by the next pass
+      CK(cudaMemsetAsync(r->group_counters, 0, sizeof(uint32_t) * need_counters, st));
+      // there is no norm step: its counters start at the value the gate|up tiles wait for
+      CK(launch_fill_u32(r->group_counters, kStackNormArrivals, static_cast<int64_t>(B) * n_blocks, st));
+      const int64_t rows = static_cast<int64_t>(n_blocks) * 256;
+      TcStackArgs a;
+      a.layers = r->recs;
+      a.n_layers = B;
+      if (!make_tmap(&a.tm_x, r->Xe, h->d, rows, h->d, 128)) return MLPMOE_ERR_CUDA;
+      if (!make_tmap_t(&a.tm_y, r->Ye, h->d, rows, h->d, 32, 4)) return MLPMOE_ERR_CUDA;
+      a.x = static_cast<float*>(r->Ye);
+      a.xnorm = r->Xe;
+      a.n = rows;
+      a.d = h->d;
+      a.bn = r->bn;
+      a.eps = 0.0f;
+      a.items = r->items;
+      a.list_offsets = r->items + n_items;
+      a.counters = r->group_counters;
+      a.status = h->status;
+      a.wait = h->wait;
+      a.out_add = 0;
+      pdl_overlap_enabled() = !h->timing;
+      CK(launch_tc_stack(a, h->num_sms, st));
+      h->launches += 2;
+    }
+    CK(launch_route_combine(r->Ye, 0, r->pos, r->rowbase, r->coef, n, B, b0, pass_end[p], h->d, p == 0, y, st));
+    h->launches += 1;
+    b0 = pass_end[p];
+  }
+  if (r->grouped) {
+    h->launches += 2;
+    return MLPMOE_OK;
+  }
   for (size_t p = 0; p < pass_end.size(); ++p) {
     for (int b = b0; b < pass_end[p]; ++b) {
       const int64_t cnt = r->counts_host[b];

@@ -82,6 +82,10 @@ cudaError_t launch_route_scan(const uint8_t* select, const uint8_t* avail, int64
                               int32_t* lists, int32_t* counts, cudaStream_t st);
 cudaError_t launch_route_coef(const int32_t* pos, int64_t n, int B, int n_avail, int compensate, float* coef, cudaStream_t st);
 cudaError_t launch_gather_rows(const void* src, const int32_t* list, int64_t n_rows, int64_t row_bytes, void* out, cudaStream_t st);
+cudaError_t launch_gather_branches(const void* src, const int32_t* lists, int64_t list_stride, const int32_t* counts,
+                                   const int32_t* rowbase, int b_lo, int b_hi, int64_t row_bytes, void* out, int blocks_per_branch,
+                                   cudaStream_t st);
+cudaError_t launch_fill_u32(uint32_t* dst, uint32_t value, int64_t count, cudaStream_t st);
 cudaError_t launch_route_combine(const void* Ye, int ye_bf16, const int32_t* pos, const int32_t* rowbase, const float* coef, int64_t n,
                                  int B, int b_lo, int b_hi, int64_t d, int first, float* y, cudaStream_t st);
 
@@ -175,6 +179,7 @@ cudaError_t launch_tc_layer(const TcLayerArgs& a, int num_sms, cudaStream_t st);
 // device memory; work items are (code, layer) pairs, code = type << 30 | column << 16 | token block.
 constexpr int kItemGateUp = 0, kItemDown = 1, kItemNorm = 2;
 constexpr int kStackNormParts = 16;    // norm items per 256-token block
+constexpr uint32_t kStackNormArrivals = kStackNormParts * 4;   // arrivals a gate|up tile waits for (2 norm warps in each CTA of the pair)
 struct alignas(64) TcStackLayer {
   CUtensorMap tm_wgu;    // Wgu [2 Ipad x d]  bf16, box 64 x 128
   CUtensorMap tm_h_st;   // H   [n x Ipad]    bf16, box 64 x 32
@@ -201,8 +206,11 @@ struct TcStackArgs {
   uint32_t* counters;            // device: [3 x n_layers x ceil(n / 256)], zero at launch
   uint32_t* status;
   WaitCfg wait;
+  int out_add = 1;               // down items accumulate into x (stack) or overwrite it (grouped branches)
 };
 cudaError_t tc_stack_init();
+void tc_stack_group_schedule(const int32_t* block_layer, int n_blocks, int64_t d, const int64_t* Ipad, int bn, int num_sms,
+                             std::vector<int32_t>* items, std::vector<int32_t>* offsets);
 void tc_stack_schedule(int64_t n, int64_t d, const int64_t* Ipad, const int* ksplit, int n_layers, int bn, int num_sms,
                        std::vector<int32_t>* items, std::vector<int32_t>* offsets);
 cudaError_t launch_tc_stack(const TcStackArgs& a, int num_sms, cudaStream_t st);

@@ -73,6 +73,27 @@ __global__ void gather_rows_kernel(const uint4* __restrict__ src, const int32_t*
   }
 }
 
+// All branches b_lo <= b < b_hi in one launch (blockIdx.y = b - b_lo): row p < counts[b] of branch b goes to row
+// rowbase[b] + p of out.  The counts are read on the device.
+__global__ void gather_branches_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ lists, int64_t list_stride,
+                                       const int32_t* __restrict__ counts, const int32_t* __restrict__ rowbase, int b_lo,
+                                       int64_t row_vecs, uint4* __restrict__ out) {
+  const int b = b_lo + blockIdx.y;
+  const int64_t total = static_cast<int64_t>(counts[b]) * row_vecs;
+  const int32_t* list = lists + static_cast<int64_t>(b) * list_stride;
+  uint4* dst = out + static_cast<int64_t>(rowbase[b]) * row_vecs;
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t r = i / row_vecs, v = i % row_vecs;
+    dst[i] = src[static_cast<int64_t>(list[r]) * row_vecs + v];
+  }
+}
+
+__global__ void fill_u32_kernel(uint32_t* __restrict__ dst, uint32_t value, int64_t count) {
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < count; i += static_cast<int64_t>(gridDim.x) * blockDim.x)
+    dst[i] = value;
+}
+
 __device__ __forceinline__ float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
 __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
   const uint2 u = *reinterpret_cast<const uint2*>(p);
@@ -126,6 +147,23 @@ cudaError_t launch_gather_rows(const void* src, const int32_t* list, int64_t n_r
   if (blocks > 148 * 16) blocks = 148 * 16;
   gather_rows_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(static_cast<const uint4*>(src), list, n_rows, row_bytes / 16,
                                                                   static_cast<uint4*>(out));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather_branches(const void* src, const int32_t* lists, int64_t list_stride, const int32_t* counts,
+                                   const int32_t* rowbase, int b_lo, int b_hi, int64_t row_bytes, void* out, int blocks_per_branch,
+                                   cudaStream_t st) {
+  if (b_hi <= b_lo) return cudaSuccess;
+  gather_branches_kernel<<<dim3(static_cast<unsigned>(blocks_per_branch), static_cast<unsigned>(b_hi - b_lo)), 256, 0, st>>>(
+      static_cast<const uint4*>(src), lists, list_stride, counts, rowbase, b_lo, row_bytes / 16, static_cast<uint4*>(out));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fill_u32(uint32_t* dst, uint32_t value, int64_t count, cudaStream_t st) {
+  if (count == 0) return cudaSuccess;
+  int64_t blocks = (count + 255) / 256;
+  if (blocks > 1024) blocks = 1024;
+  fill_u32_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(dst, value, count);
   return cudaGetLastError();
 }
 

@@ -45,6 +45,7 @@ constexpr uint32_t ARRIVALS_PER_ITEM = 8;            // 4 epilogue warps in each
 constexpr int NORM_PARTS = kStackNormParts;          // norm items per 256-token block
 constexpr uint32_t ARRIVALS_PER_NORM_ITEM = 4;       // 2 norm warps in each of the two CTAs
 constexpr int NORM_ROWS_PER_WARP = 256 / NORM_PARTS / 4;
+static_assert(NORM_PARTS * ARRIVALS_PER_NORM_ITEM == kStackNormArrivals, "the preset of the grouped-branch launches");
 constexpr int NORM_VEC = 8;                          // float4 per lane and row kept in registers (d <= 1024 in one go)
 
 struct StackParams {
@@ -62,6 +63,7 @@ struct StackParams {
   uint32_t* status;
   uint64_t wait_ns;       // limit of every bounded wait
   uint32_t extra;         // added to the target of every wait for other CTAs' arrivals (0 outside tests)
+  int out_add;            // down items add their tile into x (the residual stream) / overwrite it (grouped branches)
 };
 
 struct Item {
@@ -331,7 +333,7 @@ tc_stack_kernel(const __grid_constant__ CUtensorMap tm_x,        // Xn  [n x d] 
       if (t.type == kItemGateUp) {
         epilogue_swiglu_tma(taddr, L->scale, &L->tm_h_st, staging, tiles_stored, lane, row0, t.col * 128, release);
       } else {
-        epilogue_out_tma(taddr, &tm_y, staging, tiles_stored, lane, row0, (t.col / L->ksplit) * p.bn, p.bn, 1, release);
+        epilogue_out_tma(taddr, &tm_y, staging, tiles_stored, lane, row0, (t.col / L->ksplit) * p.bn, p.bn, p.out_add, release);
       }
       if (lane == 0) {
         tma_store_wait_all<0>();           // this warp's part of H (or of x) has been written ...
@@ -452,6 +454,63 @@ void tc_stack_schedule(int64_t n, int64_t d, const int64_t* Ipad, const int* ksp
   }
 }
 
+// Work sequences for grouped branches (per-token branch selection): every 256-row block of the
+// gathered token matrix belongs to ONE branch, whose weights are the block's "layer" record.  A
+// block has the gate|up tiles of its branch and then its down items (one K slice), nothing else:
+// no norm parts (the norm sequences are empty; the caller presets the norm counters to their
+// target) and no dependency between blocks.  Same form as tc_stack_schedule: one global order
+// (slot s: the gate|up tiles of block s, then the down items of block s - lag), dealt to the pair
+// with the least estimated work; an item only waits for items earlier in that order.
+void tc_stack_group_schedule(const int32_t* block_layer, int n_blocks, int64_t d, const int64_t* Ipad, int bn, int num_sms,
+                             std::vector<int32_t>* items, std::vector<int32_t>* offsets) {
+  const int pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
+  const int n2 = static_cast<int>((d + bn - 1) / bn);
+  const int64_t kb1 = (d + BK - 1) / BK;
+  auto kstep_cycles = [](int width) {
+    const int64_t mma = 2 * width, fill = (A_BYTES + (width / 2) * BK * 2) / 50;
+    return mma > fill ? mma : fill;
+  };
+  // (estimated work, pair) as a min-heap: this schedule is rebuilt at every call, so dealing an item costs log(pairs)
+  std::vector<std::pair<int64_t, int>> heap;
+  for (int c = 0; c < pairs; ++c) heap.emplace_back(0, c);
+  auto later = [](const std::pair<int64_t, int>& a, const std::pair<int64_t, int>& b) { return a > b; };
+  std::vector<std::vector<int32_t>> lists(pairs);
+  auto give = [&](int32_t code, int layer, int64_t cost) {
+    std::pop_heap(heap.begin(), heap.end(), later);
+    std::pair<int64_t, int>& top = heap.back();
+    lists[top.second].push_back(code);
+    lists[top.second].push_back(layer);
+    top.first += cost;
+    std::push_heap(heap.begin(), heap.end(), later);
+  };
+  // the down items of a block come about a wave and a half of gate|up tiles after the block's own tiles
+  int64_t tiles = 0;
+  for (int r = 0; r < n_blocks; ++r) tiles += Ipad[block_layer[r]] / 128;
+  const int64_t per_block = n_blocks > 0 ? (tiles + n_blocks - 1) / n_blocks : 1;
+  int lag = static_cast<int>((3 * pairs + 2 * per_block - 1) / (2 * per_block)) + 1;
+  if (lag > n_blocks) lag = n_blocks;
+  for (int sl = 0; sl < n_blocks + lag; ++sl) {
+    if (sl < n_blocks) {
+      const int l = block_layer[sl];
+      const int64_t cost_g = kb1 * kstep_cycles(256) + 1500;
+      for (int nb = 0; nb < static_cast<int>(Ipad[l] / 128); ++nb) give(encode_item(kItemGateUp, nb, sl), l, cost_g);
+    }
+    if (sl >= lag) {
+      const int r = sl - lag, l = block_layer[r];
+      const int64_t cost_d = (Ipad[l] / BK) * kstep_cycles(bn) + 1500 + 24 * bn;
+      for (int nb = 0; nb < n2; ++nb) give(encode_item(kItemDown, nb, r), l, cost_d);
+    }
+  }
+  items->clear();
+  offsets->clear();
+  offsets->push_back(0);
+  for (int c = 0; c < pairs; ++c) {
+    items->insert(items->end(), lists[c].begin(), lists[c].end());
+    offsets->push_back(static_cast<int32_t>(items->size() / 2));
+  }
+  for (int c = 0; c <= pairs; ++c) offsets->push_back(static_cast<int32_t>(items->size() / 2));    // empty norm sequences
+}
+
 cudaError_t launch_tc_stack(const TcStackArgs& a, int num_sms, cudaStream_t st) {
   if (a.n == 0 || a.n_layers == 0) return cudaSuccess;
   StackParams p{};
@@ -473,6 +532,7 @@ cudaError_t launch_tc_stack(const TcStackArgs& a, int num_sms, cudaStream_t st) 
   p.status = a.status;
   p.wait_ns = a.wait.limit_ns;
   p.extra = a.wait.extra_arrivals;
+  p.out_add = a.out_add;
   const int pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
   return launch_pdl(tc_stack_kernel, dim3(2 * pairs), dim3(STACK_THREADS), SMEM_BYTES, st, a.tm_x, a.tm_y, p);
 }
