@@ -85,6 +85,38 @@ def test_config3_structured_fade_full_size(lib):
         lib.mlpmoe_destroy(h)
 
 
+def test_config3_routed_full_size(lib):
+    """Per-token branch selection (labelled extension) at the Llama-shaped layer of configs[2], in the launch
+    configuration the bench times: 8192 tokens, every token 8 of 32 branches (2048 rows, 8 blocks per branch, 256 blocks
+    and about 5000 work items in the one grouped launch), non-unit alpha.  Rows are independent, so the oracle runs on a
+    sample of them; a second call with another selection reuses the handle's buffers."""
+    B, n, k = 32, 8192, 8
+    d_b = synth.equal_partition(I, B)
+    bits = synth.layer_weights(3, 0, D, I, 0.02, bf16=True)
+    host = [synth.bf16_bits_to_f32(b) for b in bits]
+    dev = [dev_bf16(b) for b in bits]
+    alpha = [float(np.float32(a)) for a in synth.uniform_f64((synth.BASE_SEED, 3, 0, synth.T_ALPHA), B, 0.8, 1.2)]
+    h = lib.mlpmoe_create(D, I, d_b, dev[0], dev[1], dev[2], alpha, lib.MLPMOE_BF16, lib.MLPMOE_LAYOUT_PAPER, n, stream_ptr())
+    try:
+        xb = synth.f32_to_bf16_bits(synth.tokens(3, n, D))
+        xd = dev_bf16(xb)
+        y = torch.empty((n, D), dtype=torch.float32, device="cuda")
+        rows = [0, 1, 255, 256, 3000, 4095, 4096, 8000, n - 1]
+        for trial, kk in enumerate((k, 3)):
+            sel = synth.route_select((synth.BASE_SEED, 3, trial, synth.T_ROUTE), n, B, kk)
+            sel[255] = 0
+            sel[256] = 1
+            lib.mlpmoe_forward_routed(h, xd, y, n, torch.from_numpy(sel).cuda(), True, stream_ptr())
+            torch.cuda.synchronize()
+            assert lib.mlpmoe_get_status(h) == lib.MLPMOE_OK
+            got = y.cpu().numpy()
+            ref = oracle.routed_forward(synth.bf16_bits_to_f32(xb[rows]), host[0], host[1], host[2], d_b, alpha, sel[rows])
+            assert rel_err(got[rows], ref) <= TOL_BF16
+            assert np.all(got[255] == 0.0) and np.isfinite(got).all()
+    finally:
+        lib.mlpmoe_destroy(h)
+
+
 @pytest.fixture(scope="module")
 def llama_stack():
     """Seeded bf16 weights of the 32 Llama-shaped layers: bit patterns on the host, tensors on the device."""
