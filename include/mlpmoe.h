@@ -186,11 +186,13 @@ mlpmoe_status_t mlpmoe_forward_ex(mlpmoe_handle_t h, const void* x, void* y, int
  *   y       device, [n_tokens x d_model] fp32, 16-byte aligned
  *   select  device, [n_tokens x B] row-major bytes
  * Only the selected (token, branch) pairs are computed: the tokens of a branch are
- * gathered into one block, the branch runs on it as a layer of its own (the kernels
- * of mlpmoe_forward, fp32 output), and the blocks are summed back per token in
- * ascending b.  The first call, and the first after a Fade or a prune, builds one
- * packed single-branch layer per available branch (allocates about the layer's
- * packed weights once more, plus max_tokens x min(B, 8) fp32 output rows, and
+ * gathered into a block of rows of their own, every branch runs on its block as a
+ * packed single-branch layer (bf16 layers: all branches in one launch of the
+ * persistent CTA-pair kernel; fp32 layers: one mlpmoe_forward per branch), the
+ * branch outputs stay fp32 and are summed back per token in ascending b.  The
+ * first call, and the first after a Fade or a prune, builds the single-branch
+ * layers (allocates about the layer's packed weights once more, plus input,
+ * intermediate and fp32 output rows for max_tokens x min(B, 8) selected pairs, and
  * synchronises); EVERY call synchronises `stream` once, to read the per-branch
  * token counts.  Pays for prefill-sized batches; for a handful of tokens the
  * per-branch launches cost more than the skipped branches save.

@@ -1,9 +1,10 @@
 // Per-token branch selection (dynamic routing over branches; Section 7, Limitation 2, and Section 8
 // name it as future work, the rule is this library's own and is stated in mlpmoe.h): the glue
-// around the per-branch forward calls.  Tokens are grouped by selected branch (a stable scan per
-// branch), their rows gathered into one contiguous block per branch, every branch evaluated on its
-// own block by the ordinary kernels, and the blocks' outputs summed back per token with the
-// token's compensation factor sqrt(B' / |S_t|) (Section 3.3 with K = |S_t|).  All HBM-bound.
+// around the per-branch GEMMs.  Tokens are grouped by selected branch (a stable scan per branch),
+// their rows gathered into one contiguous block per branch, every branch evaluated on its own
+// block by the layer kernels (bf16: all blocks in one launch of the stack kernel, the branches as
+// its layer records), and the blocks' outputs summed back per token with the token's compensation
+// factor sqrt(B' / |S_t|) (Section 3.3 with K = |S_t|).  All HBM-bound.
 #include "internal.h"
 
 namespace mlpmoe {
