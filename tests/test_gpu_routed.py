@@ -1,8 +1,9 @@
 """GPU parity of mlpmoe_forward_routed (per-token branch selection, a labelled extension: the paper
 names dynamic routing over branches as future work only) against oracle.routed_forward, element by
-element through the C ABI: token counts per branch that land in every kernel family (decode pair,
-single-CTA GEMM pair, fused CTA-pair kernel), tokens that select nothing, branches nobody selects,
-unavailable branches, several output passes, Fade and pruning before routing, fp32."""
+element through the C ABI: bf16 layers (all branches in one launch of the stack kernel) and fp32
+layers (one layer call per branch, with token counts that land in each of its kernel families),
+tokens that select nothing, branches nobody selects, unavailable branches, several output passes,
+Fade and pruning before routing."""
 import numpy as np
 import pytest
 import torch
@@ -27,8 +28,8 @@ def run_routed(lib, h, xd, sel, n, d, compensate=True):
 @pytest.mark.parametrize("bf16", [True, False])
 @pytest.mark.parametrize("n,k", [(1, 2), (13, 1), (70, 2), (300, 3), (700, 2)])
 def test_small_layer_routed(lib, bf16, n, k):
-    """d = 320, unequal branches (one of 16 neurons), non-unit alpha with a negative gate.  700 tokens with 2 of 5
-    branches put about 280 tokens on a branch (fused pair kernel), 300 x 3/5 = 180, 70 x 2/5 = 28 (decode pair)."""
+    """d = 320, unequal branches (one of 16 neurons, so the padded widths differ), non-unit alpha with a negative gate.
+    700 tokens with 2 of 5 branches put about 280 tokens (two 256-row blocks) on a branch, 300 x 3/5 = 180, 70 x 2/5 = 28."""
     d, d_b = 320, [64, 160, 16, 160, 112]
     I = sum(d_b)
     alpha = [1.0, 0.8, 1.2, -0.5, 0.9]
@@ -50,27 +51,30 @@ def test_small_layer_routed(lib, bf16, n, k):
         lib.mlpmoe_destroy(h)
 
 
-def test_every_branch_selected_equals_forward_and_passes(lib):
-    """B = 12 > 8 branches all selected by all tokens: the branch outputs need two passes through the output buffer;
-    the result is the plain layer (Section 3.1) at the bf16 tolerance."""
+@pytest.mark.parametrize("bf16", [True, False])
+def test_every_branch_selected_equals_forward_and_passes(lib, bf16):
+    """B = 12 > 8 branches all selected by all 1024 = max_tokens tokens: 12 x 1024 selected rows against room for
+    8 x 1024 + 12 x 256, so the branch outputs take two passes through the buffers; the result is the plain layer
+    (Section 3.1) at the bf16 tolerance."""
     d, B = 256, 12
     d_b = [32] * B
-    c = Case((301,), d, 32 * B, d_b, bf16=True, std=0.05, alpha=list(np.linspace(0.7, 1.3, B)))
-    n = 200
+    c = Case((301,), d, 32 * B, d_b, bf16=bf16, std=0.05, alpha=list(np.linspace(0.7, 1.3, B)))
+    tol = TOL_BF16 if bf16 else TOL_FP32
+    n = 1024
     xh, xd = c.tokens((301,), n)
     h = c.create(lib, n)
     try:
         sel = np.ones((n, B), dtype=np.uint8)
         y = run_routed(lib, h, xd, sel, n, d)
         ref = oracle.mlpmoe_forward(xh, *c.host, d_b, c.alpha)
-        assert rel_err(y, ref) <= TOL_BF16
+        assert rel_err(y, ref) <= tol
         # a routing that leaves branches 3 and 7 to nobody
         sel2 = synth.route_select((301, synth.T_ROUTE), n, B, 5)
         sel2[:, 3] = 0
         sel2[:, 7] = 0
         y2 = run_routed(lib, h, xd, sel2, n, d)
         ref2 = oracle.routed_forward(xh, *c.host, d_b, c.alpha, sel2)
-        assert rel_err(y2, ref2) <= TOL_BF16
+        assert rel_err(y2, ref2) <= tol
     finally:
         lib.mlpmoe_destroy(h)
 
