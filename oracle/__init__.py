@@ -8,6 +8,7 @@ from .mlpmoe_oracle import (  # noqa: F401
     silu,
     branch_forward,
     mlpmoe_forward,
+    mlpmoe_forward_h_bf16,
     routed_forward,
     fade_schedule,
     fade_position,

@@ -247,6 +247,31 @@ def prune_alpha(alpha: Sequence[float], keep: Sequence[bool], compensate: bool =
     return [float(alpha[b]) * c if keep[b] else 0.0 for b in range(B)]
 
 
+def mlpmoe_forward_h_bf16(x, W_gate, W_up, W_down, d_b: Sequence[int],
+                          alpha: Optional[Sequence[float]] = None) -> np.ndarray:
+    """The layer equation of Section 3.1 with ONE rounding added, the one a bf16
+    implementation that keeps the intermediate in bf16 commits: per branch
+    h = bf16(alpha_b * phi(W_gate^(b) x) (.) W_up^(b) x), then y = sum_b W_down^(b) h.
+    Everything else stays float64.  Not the paper's arithmetic (the paper fixes no
+    precision): a model of the stated storage format, used to check a bf16 kernel
+    far more tightly than the paper-level tolerance allows.  |y - mlpmoe_forward|
+    is bounded by 2^-9 * sum_j |h_j W_down[j, m]| (half an ulp per h)."""
+    x = np.asarray(x, dtype=np.float64)
+    d, I = np.asarray(W_gate).shape
+    offs = branch_offsets(d_b, I)
+    B = len(d_b)
+    if alpha is None:
+        alpha = [1.0] * B
+    y = np.zeros((x.shape[0], d), dtype=np.float64)
+    for b in range(B):
+        lo, hi = offs[b], offs[b + 1]
+        g = x @ np.asarray(W_gate)[:, lo:hi].astype(np.float64)
+        u = x @ np.asarray(W_up)[:, lo:hi].astype(np.float64)
+        h = round_to_bf16(float(alpha[b]) * (silu(g) * u))
+        y = y + h @ np.asarray(W_down)[lo:hi, :].astype(np.float64)
+    return y
+
+
 def routed_forward(x, W_gate, W_up, W_down, d_b: Sequence[int], alpha: Sequence[float], select,
                    compensate: bool = True) -> np.ndarray:
     """Per-token branch selection, a labelled extension (NOT defined by the paper:

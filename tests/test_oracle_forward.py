@@ -195,3 +195,24 @@ def test_planted_mistakes_are_caught(monkeypatch):
     assert not _pins_hold()
     monkeypatch.undo()
     assert _pins_hold()
+
+
+def test_bf16_intermediate_model_is_the_layer_plus_one_rounding():
+    """mlpmoe_forward_h_bf16 (a model of a bf16 implementation's stored intermediate, not the paper's
+    arithmetic): the rounding is done here by another library (torch's bfloat16 conversion), the
+    result must agree exactly; and it stays within half a bf16 ulp per h of the unrounded layer."""
+    rng = np.random.default_rng(11)
+    d, d_b = 12, [16, 32, 16]
+    I = sum(d_b)
+    x, Wg, Wu, Wd = rng.normal(size=(9, d)), rng.normal(size=(d, I)), rng.normal(size=(d, I)), rng.normal(size=(I, d))
+    alpha = [1.0, 0.7, 1.9]
+    got = oracle.mlpmoe_forward_h_bf16(x, Wg, Wu, Wd, d_b, alpha)
+    g, u = x @ Wg, x @ Wu
+    scale = np.repeat(alpha, d_b)
+    h = g / (1.0 + np.exp(-g)) * u * scale
+    hb = torch.from_numpy(h.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    np.testing.assert_allclose(got, hb @ Wd, rtol=1e-13, atol=1e-13)
+    plain = oracle.mlpmoe_forward(x, Wg, Wu, Wd, d_b, alpha)
+    bound = 2.0 ** -9 * (np.abs(h) @ np.abs(Wd))
+    assert np.all(np.abs(got - plain) <= bound + 1e-12)
+    assert np.abs(got - plain).max() > 0          # the rounding is really there
