@@ -300,6 +300,45 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ 
   }
 }
 
+// One warp per token row with the whole row in registers (d <= 128 NV): every load of the row is in
+// flight before the first use, and the row crosses the memory system once.  The sum of squares adds
+// the same terms in the same order as rmsnorm_kernel.
+template <bool OUT_BF16, int NV>
+__global__ void __launch_bounds__(256) rmsnorm_reg_kernel(const float* __restrict__ x, void* __restrict__ r, int64_t n,
+                                                          int64_t d, float eps) {
+  const int64_t t = static_cast<int64_t>(blockIdx.x) * (blockDim.x / 32) + threadIdx.x / 32;
+  const int lane = threadIdx.x % 32;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (t >= n) return;
+  const float4* row = reinterpret_cast<const float4*>(x + t * d);
+  const int64_t nv = d / 4;
+  float4 a[NV];
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int64_t v = static_cast<int64_t>(i) * 32 + lane;
+    a[i] = v < nv ? __ldcs(row + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) ss += a[i].x * a[i].x + a[i].y * a[i].y + a[i].z * a[i].z + a[i].w * a[i].w;
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+  const float inv = 1.0f / sqrtf(ss / static_cast<float>(d) + eps);
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int64_t v = static_cast<int64_t>(i) * 32 + lane;
+    if (v >= nv) continue;
+    if (OUT_BF16) {
+      uint2 o;
+      o.x = static_cast<uint32_t>(f32_to_bf16_rn(a[i].x * inv)) | (static_cast<uint32_t>(f32_to_bf16_rn(a[i].y * inv)) << 16);
+      o.y = static_cast<uint32_t>(f32_to_bf16_rn(a[i].z * inv)) | (static_cast<uint32_t>(f32_to_bf16_rn(a[i].w * inv)) << 16);
+      reinterpret_cast<uint2*>(static_cast<uint16_t*>(r) + t * d)[v] = o;
+    } else {
+      reinterpret_cast<float4*>(static_cast<float*>(r) + t * d)[v] = make_float4(a[i].x * inv, a[i].y * inv, a[i].z * inv, a[i].w * inv);
+    }
+  }
+}
+
 // Few rows (decode): one 256-thread block per row, so that a row's loads are all in flight at once.
 template <bool OUT_BF16>
 __global__ void __launch_bounds__(256) rmsnorm_block_kernel(const float* __restrict__ x, void* __restrict__ r, int64_t n,
@@ -461,6 +500,10 @@ cudaError_t launch_rmsnorm(const float* x, void* r, int64_t n, int64_t d, float 
       return launch_pdl(rmsnorm_block_kernel<true>, dim3(static_cast<unsigned>(n)), dim3(256), 0, st, x, r, n, d, eps);
     return launch_pdl(rmsnorm_block_kernel<false>, dim3(static_cast<unsigned>(n)), dim3(256), 0, st, x, r, n, d, eps);
   }
+  if (out_elem_size == 2 && d <= 1024)
+    return launch_pdl(rmsnorm_reg_kernel<true, 8>, dim3(cdiv(n, 8)), dim3(256), 0, st, x, r, n, d, eps);
+  if (out_elem_size == 2 && d <= 4096)
+    return launch_pdl(rmsnorm_reg_kernel<true, 32>, dim3(cdiv(n, 8)), dim3(256), 0, st, x, r, n, d, eps);
   if (out_elem_size == 2)
     return launch_pdl(rmsnorm_kernel<true>, dim3(cdiv(n, 8)), dim3(256), 0, st, x, r, n, d, eps);
   return launch_pdl(rmsnorm_kernel<false>, dim3(cdiv(n, 8)), dim3(256), 0, st, x, r, n, d, eps);
