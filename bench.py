@@ -106,7 +106,7 @@ TRAFFIC = {
     # workload key: (bytes per launch, source files, sha256[:16] of their concatenation, profile)
     "llama_prefill": ((6234150144 + 627657728 + 5631617792 + 619579904) / 2, ('tc_layer.cu', 'tc_common.cuh', 'ptx.cuh'), "61d5a0e50491c749",
                       "profiles/tc_layer_kernel_llama_c5_16384tokens.md (mean of the two layers captured at the headline shape)"),
-    "qwen_stack": (861574656 + 955400960, ('tc_stack.cu', 'tc_common.cuh', 'ptx.cuh'), "f920260a14cffc56", "profiles/tc_stack_kernel_qwen_c2_24layers.md"),
+    "qwen_stack": (865387520 + 955156480, ('tc_stack.cu', 'tc_common.cuh', 'ptx.cuh'), "8fb514fda6c30732", "profiles/tc_stack_kernel_qwen_c2_24layers.md"),
     # decode: captured on 4 of the 32 layers; a launch streams its layers' weights once, so traffic scales with the layers
     "llama_decode_1": ((1470823936 + 4195840) * 8, ('decode_fused.cu', 'ptx.cuh'), "41ae9186018dac22", "profiles/decode_fused_kernel_llama_c4_4layers.md"),
     "llama_decode_8": ((1467553280 + 4698368) * 8, ('decode_fused.cu', 'ptx.cuh'), "41ae9186018dac22", "profiles/decode_fused_kernel_llama_c4_4layers.md"),
