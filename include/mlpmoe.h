@@ -417,6 +417,17 @@ mlpmoe_status_t mlpmoe_host_stack_schedule(int64_t n_tokens, int64_t d_model, in
                                            const int32_t* ksplit, int32_t bn, int32_t num_sms, int32_t* items,
                                            int64_t item_capacity, int64_t* n_items, int32_t* offsets);
 
+/*
+ * The work sequences of the one grouped launch of mlpmoe_forward_routed on a bf16 layer (set-up logic, no
+ * CUDA call): block r of the gathered token rows (256 rows) belongs to branch block_branch[r] and has that
+ * branch's n_active_pad[b]/128 gate|up tiles and ceil(d_model/bn) down items, nothing else.  items, n_items and
+ * the GEMM half of offsets as in mlpmoe_host_stack_schedule, the second int32 of an item being the branch
+ * and the token-block field the block index r; the norm sequences (second half of offsets) are empty.
+ */
+mlpmoe_status_t mlpmoe_host_group_schedule(const int32_t* block_branch, int32_t n_blocks, int64_t d_model, int32_t n_branches,
+                                           const int64_t* n_active_pad, int32_t bn, int32_t num_sms, int32_t* items,
+                                           int64_t item_capacity, int64_t* n_items, int32_t* offsets);
+
 #ifdef __cplusplus
 }
 #endif

@@ -73,6 +73,8 @@ SIGNATURES = {
                                             POINTER(c_int32)]),
     "mlpmoe_host_stack_schedule": (c_int32, [c_int64, c_int64, c_int32, POINTER(c_int64), POINTER(c_int32), c_int32, c_int32,
                                              POINTER(c_int32), c_int64, POINTER(c_int64), POINTER(c_int32)]),
+    "mlpmoe_host_group_schedule": (c_int32, [POINTER(c_int32), c_int32, c_int64, c_int32, POINTER(c_int64), c_int32, c_int32,
+                                             POINTER(c_int32), c_int64, POINTER(c_int64), POINTER(c_int32)]),
     "mlpmoe_host_schedule": (c_int32, [c_int32, POINTER(c_int64), POINTER(c_float), POINTER(c_uint8), POINTER(c_int32),
                                        POINTER(c_int32), POINTER(c_int64), POINTER(c_int64), POINTER(c_int32),
                                        POINTER(c_int64)]),
@@ -362,3 +364,20 @@ def mlpmoe_host_stack_schedule(n_tokens: int, d_model: int, n_active_pad: Sequen
     gemm = [seq(offs[c], offs[c + 1]) for c in range(pairs)]
     norm = [seq(offs[pairs + 1 + c], offs[pairs + 2 + c]) for c in range(pairs)]
     return gemm, norm
+
+
+def mlpmoe_host_group_schedule(block_branch: Sequence[int], d_model: int, n_active_pad: Sequence[int], bn: int, num_sms: int = 148):
+    """For each CTA pair its sequence of items (type, column, block, branch) of the grouped launch of the routed
+    forward; type 0 = gate|up tile, 1 = down item."""
+    nb, B = len(block_branch), len(n_active_pad)
+    pairs = num_sms // 2
+    n2 = (d_model + bn - 1) // bn
+    cap = sum(n_active_pad[b] // 128 + n2 for b in block_branch) + 1
+    items = (c_int32 * (2 * cap))()
+    n_items = c_int64()
+    offs = (c_int32 * (2 * (pairs + 1)))()
+    _check(lib.mlpmoe_host_group_schedule((c_int32 * max(nb, 1))(*block_branch), nb, d_model, B, (c_int64 * B)(*n_active_pad), bn, num_sms,
+                                          items, cap, ctypes.byref(n_items), offs), "mlpmoe_host_group_schedule")
+    assert all(offs[pairs + 1 + c] == n_items.value for c in range(pairs + 1))      # the norm sequences are empty
+    return [[((items[2 * i] >> 30) & 3, (items[2 * i] >> 16) & 0x3FFF, items[2 * i] & 0xFFFF, items[2 * i + 1])
+             for i in range(offs[c], offs[c + 1])] for c in range(pairs)]

@@ -1517,4 +1517,23 @@ mlpmoe_status_t mlpmoe_host_stack_schedule(int64_t n_tokens, int64_t d_model, in
   return MLPMOE_OK;
 }
 
+mlpmoe_status_t mlpmoe_host_group_schedule(const int32_t* block_branch, int32_t n_blocks, int64_t d_model, int32_t n_branches,
+                                           const int64_t* n_active_pad, int32_t bn, int32_t num_sms, int32_t* items,
+                                           int64_t item_capacity, int64_t* n_items, int32_t* offsets) {
+  if (!block_branch || n_blocks < 0 || d_model <= 0 || n_branches <= 0 || !n_active_pad || bn < 32 || bn > 256 || bn % 32 != 0 ||
+      num_sms < 2 || !items || !n_items || !offsets)
+    return MLPMOE_ERR_INVALID_ARG;
+  for (int b = 0; b < n_branches; ++b)
+    if (n_active_pad[b] <= 0 || n_active_pad[b] % 128 != 0) return MLPMOE_ERR_INVALID_ARG;
+  for (int r = 0; r < n_blocks; ++r)
+    if (block_branch[r] < 0 || block_branch[r] >= n_branches) return MLPMOE_ERR_INVALID_ARG;
+  std::vector<int32_t> t, o;
+  tc_stack_group_schedule(block_branch, n_blocks, d_model, n_active_pad, bn, num_sms, &t, &o);
+  *n_items = static_cast<int64_t>(t.size() / 2);
+  if (static_cast<int64_t>(t.size() / 2) > item_capacity) return MLPMOE_ERR_INVALID_ARG;
+  std::memcpy(items, t.data(), sizeof(int32_t) * t.size());
+  std::memcpy(offsets, o.data(), sizeof(int32_t) * o.size());
+  return MLPMOE_OK;
+}
+
 }  // extern "C"

@@ -236,3 +236,38 @@ def test_stack_schedule_is_complete_and_cannot_deadlock(lib, n, d, Ipads, kss, b
     counts = [len(lst) for lst in gemm]
     if len(flat) >= 8 * 74:
         assert max(counts) <= 1.5 * (sum(counts) / len(counts)) + 4
+
+
+@pytest.mark.parametrize("blocks,d,Ipads,bn", [([0] * 8 + [1] * 3 + [3] * 9, 4096, [512, 512, 384, 512], 256),
+                                                ([2, 0, 0, 1], 320, [128, 256, 128], 160),
+                                                (sum(([b] * 8 for b in range(32)), []), 4096, [512] * 32, 256), ([], 256, [128], 128)])
+def test_group_schedule_is_complete_and_cannot_deadlock(lib, blocks, d, Ipads, bn):
+    """The one grouped launch of the routed forward: every block has exactly its branch's gate|up tiles and its down
+    items, once; a down item waits for all gate|up tiles of its block and nothing else waits; whatever the items' real
+    durations, running the pairs' sequences under that rule finishes; the items are spread evenly."""
+    lists = lib.mlpmoe_host_group_schedule(blocks, d, Ipads, bn, 148)
+    n2 = (d + bn - 1) // bn
+    want = set()
+    for r, b in enumerate(blocks):
+        want |= {(0, nb, r, b) for nb in range(Ipads[b] // 128)}
+        want |= {(1, nb, r, b) for nb in range(n2)}
+    flat = [t for lst in lists for t in lst]
+    assert len(flat) == len(set(flat)) and set(flat) == want
+    rng = np.random.default_rng(len(blocks))
+    for trial in range(2):
+        pos = [0] * len(lists)
+        tiles_done = {}
+        remaining = len(flat)
+        while remaining:
+            runnable = [c for c in range(len(lists)) if pos[c] < len(lists[c]) and
+                        (lists[c][pos[c]][0] == 0 or tiles_done.get(lists[c][pos[c]][2], 0) == Ipads[lists[c][pos[c]][3]] // 128)]
+            assert runnable, "every pair is blocked: the schedule can deadlock"
+            for c in rng.permutation(runnable)[: max(1, len(runnable) // 2)]:
+                t = lists[c][pos[c]]
+                if t[0] == 0:
+                    tiles_done[t[2]] = tiles_done.get(t[2], 0) + 1
+                pos[c] += 1
+                remaining -= 1
+    if len(flat) >= 8 * 74:
+        cost = [sum(64 * 512 if t[0] == 0 else Ipads[t[3]] // 64 * 2 * bn for t in lst) for lst in lists]
+        assert max(cost) <= 1.1 * (sum(cost) / len(cost)) + 64 * 512
