@@ -176,6 +176,7 @@ struct Routed {
   int64_t counters_cap = 0;
   std::vector<int32_t> items_host, block_layer;
   std::vector<int64_t> ipad_host;
+  Workspace* no_ws = nullptr;              // what the per-branch layers share in grouped mode: sizes only, no memory
 };
 
 }  // namespace
@@ -270,6 +271,7 @@ void free_routed(Routed* r) {
   for (mlpmoe_layer_s* c : r->child) free_layer(c);
   cudaFree(r->avail); cudaFree(r->pos); cudaFree(r->lists); cudaFree(r->counts); cudaFree(r->rowbase); cudaFree(r->coef);
   cudaFree(r->Xe); cudaFree(r->Ye); cudaFree(r->recs); cudaFree(r->Hg); cudaFree(r->items); cudaFree(r->group_counters);
+  ws_release(r->no_ws);
   delete r;
 }
 
@@ -884,6 +886,19 @@ mlpmoe_status_t ensure_routed(mlpmoe_layer_s* h, cudaStream_t st) {
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return h->d_b[a] > h->d_b[b]; });
   r->n_avail = static_cast<int>(order.size());
   Workspace* ws = nullptr;
+  if (r->grouped) {
+    // the grouped launch has its own buffers (Xe, Hg, Ye): the per-branch layers get a workspace without memory
+    if (!r->no_ws) {
+      r->no_ws = new (std::nothrow) Workspace();
+      if (!r->no_ws) return MLPMOE_ERR_ALLOC;
+      r->no_ws->refs = 1;
+      r->no_ws->max_tokens = h->max_tokens;
+      r->no_ws->Ipad_max = h->Ipad_max;
+      r->no_ws->d = h->d;
+      r->no_ws->elem_size = h->elem_size;
+    }
+    ws = r->no_ws;
+  }
   const size_t row = static_cast<size_t>(h->d) * h->elem_size;
   for (int b : order) {
     const size_t off = static_cast<size_t>(h->offs[b]) * row;
