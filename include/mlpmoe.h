@@ -328,6 +328,15 @@ mlpmoe_status_t mlpmoe_get_timing(mlpmoe_handle_t h, double* ms, int64_t* launch
 mlpmoe_status_t mlpmoe_debug_set_wait(mlpmoe_handle_t h, uint64_t limit_ns, uint32_t extra_arrivals);
 
 /*
+ * Which persistent kernel a decode stack call (at most 64 tokens) that starts with this layer runs:
+ * 0 = by the library's rule (token count and how many SMs own a neuron tile), 1 = the few-token kernel
+ * (both GEMMs on the tile's owner; at most 16 tokens, more tokens fall back to the rule's other kernel),
+ * 2 = the kernel with a grid-wide H exchange.  Both compute the same stack; the tests use this to run
+ * each of them on shapes where the rule would pick the other.  MLPMOE_ERR_INVALID_ARG for another value.
+ */
+mlpmoe_status_t mlpmoe_debug_set_decode_kernel(mlpmoe_handle_t h, int32_t kernel);
+
+/*
  * The handle's (possibly shared) activation workspace, for guard-band checks and memory
  * accounting: device addresses and sizes in bytes of H (n x n_active_pad of the layer dtype for
  * an n-token call), of the normalised / staged input (n x d_model, layer dtype) and of the fp32

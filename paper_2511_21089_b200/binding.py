@@ -49,6 +49,7 @@ SIGNATURES = {
     "mlpmoe_rmsnorm": (c_int32, [c_void_p, c_void_p, c_int64, c_int64, c_float, c_int32, c_void_p]),
     "mlpmoe_stack_prepare": (c_int32, [POINTER(c_void_p), c_int32, c_int64, c_void_p]),
     "mlpmoe_debug_set_wait": (c_int32, [c_void_p, ctypes.c_uint64, ctypes.c_uint32]),
+    "mlpmoe_debug_set_decode_kernel": (c_int32, [c_void_p, c_int32]),
     "mlpmoe_get_workspace": (c_int32, [c_void_p, POINTER(c_void_p), POINTER(c_int64), POINTER(c_void_p), POINTER(c_int64),
                                        POINTER(c_void_p), POINTER(c_int64), POINTER(c_int64)]),
     "mlpmoe_stack_forward": (c_int32, [POINTER(c_void_p), c_int32, c_void_p, c_int64, c_float, c_void_p]),
@@ -197,6 +198,10 @@ def mlpmoe_stack_forward(layers: Sequence[int], x, n_tokens: int, eps: float = 1
 def mlpmoe_stack_prepare(layers: Sequence[int], n_tokens: int, stream=None) -> None:
     arr = (c_void_p * len(layers))(*layers)
     _check(lib.mlpmoe_stack_prepare(arr, len(layers), n_tokens, _stream(stream)), "mlpmoe_stack_prepare")
+
+
+def mlpmoe_debug_set_decode_kernel(h: int, kernel: int) -> None:
+    _check(lib.mlpmoe_debug_set_decode_kernel(h, kernel), "mlpmoe_debug_set_decode_kernel")
 
 
 def mlpmoe_debug_set_wait(h: int, limit_ns: int = 0, extra_arrivals: int = 0) -> None:

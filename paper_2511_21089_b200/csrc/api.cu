@@ -222,6 +222,7 @@ struct mlpmoe_layer_s {
   int plan_npad = 0;
   CUtensorMap plan_tm_x;                                    // normalised rows [n x d] as the kernels' token operand
   WaitCfg wait;                                             // bounded-wait limits of this handle's launches (test hook)
+  int decode_kernel = 0;                                    // test hook: 0 = by rule, 1 = few-token kernel, 2 = the 14..64-token kernel
   // fast fp32 mode (fp32 layers): three-way bf16 splits of the packed operands and of the activations
   bool fast32 = false;
   int64_t dp = 0;                                           // d rounded up to the 64-wide K-step
@@ -583,7 +584,17 @@ mlpmoe_status_t plan_decode(const mlpmoe_handle_t* layers, int32_t n_layers, int
   }
   CK(cudaMemcpyAsync(h0->stack_dev, h0->stack_host.data(), sizeof(DecodeStackLayer) * h0->stack_host.size(), cudaMemcpyHostToDevice, st));
   if (!make_tmap(&h0->plan_tm_x, h0->ws->xnorm, h0->d, n, h0->d, npad)) return MLPMOE_ERR_CUDA;
-  h0->plan_fused = tiled && n <= kDecodeFusedMaxTokens;
+  // Which of the two decode kernels: the few-token kernel keeps both GEMMs of a neuron tile on the tile's owner, so with
+  // few tiles (pruned stacks) few SMs do all the work, while the other kernel spreads its down phase over all SMs.
+  // Measured crossovers on 4096 x 14336 layers (tiles per layer over SMs: tokens up to which the few-token kernel wins):
+  // 112/148: 13, 102/148: 12, 90/148 and 70/148: 7, 56/148 and below: none.
+  int64_t tiles = 0;
+  for (int l = 0; l < n_layers; ++l) tiles += layers[l]->Ipad / 128;
+  const double owners = static_cast<double>(tiles) / n_layers / h0->num_sms;
+  int fused_max = owners > 0.71 ? kDecodeFusedMaxTokens : (owners > 0.64 ? 12 : (owners > 0.38 ? 7 : 0));
+  if (h0->decode_kernel == 1) fused_max = 16;              // the few-token kernel holds 16 token rows
+  if (h0->decode_kernel == 2) fused_max = 0;
+  h0->plan_fused = tiled && n <= fused_max;
   h0->plan_npad = npad;
   return MLPMOE_OK;
 }
@@ -1375,6 +1386,14 @@ mlpmoe_status_t mlpmoe_get_status(mlpmoe_handle_t h) {
   CK(cudaMemset(h->counters, 0, sizeof(uint32_t) * ((h->d + 127) / 128) * 4));
   CK(cudaMemset(h->status, 0, sizeof(uint32_t)));
   return MLPMOE_ERR_DEVICE_TIMEOUT;
+}
+
+mlpmoe_status_t mlpmoe_debug_set_decode_kernel(mlpmoe_handle_t h, int32_t kernel) {
+  if (!h || kernel < 0 || kernel > 2) return MLPMOE_ERR_INVALID_ARG;
+  h->decode_kernel = kernel;
+  h->plan_kind = PLAN_NONE;            // the next stack call chooses again
+  h->plan_key.clear();
+  return MLPMOE_OK;
 }
 
 mlpmoe_status_t mlpmoe_debug_set_wait(mlpmoe_handle_t h, uint64_t limit_ns, uint32_t extra_arrivals) {

@@ -56,8 +56,8 @@ def test_odd_width_layer_with_guard_bands(lib, n):
         lib.mlpmoe_destroy(h)
 
 
-@pytest.mark.parametrize("n", TOKEN_COUNTS)
-def test_odd_width_stack_with_guard_bands(lib, n):
+@pytest.mark.parametrize("n,kernel", [(n, 0) for n in TOKEN_COUNTS] + [(1, 1), (13, 1)])
+def test_odd_width_stack_with_guard_bands(lib, n, kernel):
     """Three layers with d_model = 328 as a pre-norm stack (decode-fused, decode-stack, 65..128-token and
     prefill-stack kernels by token count), the residual stream between guard bands, the workspace poisoned."""
     d, I, d_b, L = 328, 384, [128, 64, 192], 3
@@ -70,6 +70,7 @@ def test_odd_width_stack_with_guard_bands(lib, n):
                 lib.mlpmoe_share_workspace(h, handles[0])
             handles.append(h)
             layers.append((*c.host, d_b, c.alpha))
+        lib.mlpmoe_debug_set_decode_kernel(handles[0], kernel)      # 1: the few-token kernel (the rule picks the other one on layers this small)
         x = synth.normal_f32((401, 9, n), (n, d), 1.0)
         ref = oracle.stack_forward(x, layers, bf16_activations=True)
         lib.mlpmoe_stack_prepare(handles, n, stream_ptr())
@@ -136,8 +137,8 @@ def test_single_branch_and_narrow_survivors(lib, bf16, n):
         lib.mlpmoe_destroy(h)
 
 
-@pytest.mark.parametrize("n,stack", [(4, True), (40, True), (300, True), (300, False)])
-def test_bounded_wait_runs_out_and_the_handle_recovers(lib, n, stack):
+@pytest.mark.parametrize("n,stack,kernel", [(4, True, 1), (4, True, 2), (40, True, 0), (300, True, 0), (300, False, 0)])
+def test_bounded_wait_runs_out_and_the_handle_recovers(lib, n, stack, kernel):
     """The give-up path of the kernels whose CTAs wait for one another (few-token decode stack, 14..64-token
     decode stack, prefill stack, single-layer prefill): with the wait limit cut to 3 ms and every
     cross-CTA target raised by one arrival (a count that is never reached) the call must return, the
@@ -154,6 +155,7 @@ def test_bounded_wait_runs_out_and_the_handle_recovers(lib, n, stack):
             cases.append(c)
             handles.append(h)
         ones = [1.0] * len(d_b)
+        lib.mlpmoe_debug_set_decode_kernel(handles[0], kernel)
         if stack:
             x = synth.normal_f32((404, 9, n), (n, d), 1.0)
             ref = oracle.stack_forward(x, [(*c.host, d_b, ones) for c in cases], bf16_activations=True)

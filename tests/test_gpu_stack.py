@@ -28,9 +28,15 @@ def test_rmsnorm_kernel(lib):
     assert np.mean(got != oracle.round_to_bf16(ref)) < 1e-3
 
 
-@pytest.mark.parametrize("bf16", [True, False])
-@pytest.mark.parametrize("n", [1, 5, 12, 13, 14, 24, 64, 100, 129, 300, 512])
-def test_small_stack(lib, bf16, n):
+# (tokens, decode kernel): 1 = the few-token kernel, 2 = the kernel with the H exchange, 0 = the library's rule
+# (on layers as small as these the rule always picks kernel 2 for at most 64 tokens)
+SMALL_STACK_CASES = [(1, 1), (1, 2), (5, 1), (5, 2), (12, 1), (13, 1), (13, 2), (16, 1), (14, 0), (24, 0), (64, 0), (100, 0), (129, 0),
+                     (300, 0), (512, 0)]
+
+
+@pytest.mark.parametrize("bf16,n,kernel", [(True, n, k) for n, k in SMALL_STACK_CASES] +
+                         [(False, n, 0) for n in sorted({n for n, _ in SMALL_STACK_CASES})])
+def test_small_stack(lib, bf16, n, kernel):
     d, I, d_b, L = 256, 384, [128, 64, 192], 3
     cases, handles, layers = [], [], []
     try:
@@ -43,6 +49,7 @@ def test_small_stack(lib, bf16, n):
                 lib.mlpmoe_share_workspace(h, handles[0])
             handles.append(h)
             layers.append((*c.host, d_b, oracle.prune_alpha(c.alpha, keep)))
+        lib.mlpmoe_debug_set_decode_kernel(handles[0], kernel)
         x = synth.normal_f32((201, 9, n), (n, d), 1.0)
         xd = dev_f32(x)
         lib.mlpmoe_stack_forward(handles, xd, n, 1e-6, stream_ptr())
@@ -168,8 +175,8 @@ def test_two_full_width_layers_every_row(lib):
             lib.mlpmoe_destroy(h)
 
 
-@pytest.mark.parametrize("n", [4, 40, 300])
-def test_stack_follows_a_later_prune_and_fade(lib, n):
+@pytest.mark.parametrize("n,kernel", [(4, 1), (4, 2), (40, 0), (300, 0)])
+def test_stack_follows_a_later_prune_and_fade(lib, n, kernel):
     """The stack kernels cache per-stack set-up (work sequences, layer records, the decode kernel's
     tiled weight copy): a prune or a Fade between two calls must show in the second call."""
     d, I, d_b, L = 256, 512, [128, 128, 64, 192], 2
@@ -182,6 +189,7 @@ def test_stack_follows_a_later_prune_and_fade(lib, n):
                 lib.mlpmoe_share_workspace(h, handles[0])
             cases.append(c)
             handles.append(h)
+        lib.mlpmoe_debug_set_decode_kernel(handles[0], kernel)
         x = synth.normal_f32((207, 9, n), (n, d), 1.0)
         ones = [1.0] * len(d_b)
 
