@@ -477,7 +477,10 @@ class Bench:
             share = float(kms[0] / ms_timed)
             if n <= 64 and w["stack"]:
                 achieved = sum(wbytes) / (main_ms * 1e-3) / 1e9
-                kernel = ("decode_fused_kernel" if n <= 13 else "decode_stack_kernel") + \
+                # the library's rule (plan_decode): the few-token kernel up to 13 tokens, fewer when few SMs own a neuron tile
+                owners = float(np.mean([(a + 127) // 128 for a in active])) / self.torch.cuda.get_device_properties(0).multi_processor_count
+                fused_max = 13 if owners > 0.71 else (12 if owners > 0.64 else (7 if owners > 0.38 else 0))
+                kernel = ("decode_fused_kernel" if n <= fused_max else "decode_stack_kernel") + \
                     ": whole stack in one persistent launch (bulk-copy weight ring + tcgen05)"
                 out["roofline"] = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
                                    "frac": achieved / pk["hbm_gbs"], "traffic": traffic_for(w),
