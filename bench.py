@@ -475,7 +475,7 @@ class Bench:
             ms_timed = ms_total * timed_steps / steps
             main_ms = kms[0] / kcnt[0]
             share = float(kms[0] / ms_timed)
-            if n <= 64 and w["stack"]:
+            if n <= 128 and w["stack"]:
                 achieved = sum(wbytes) / (main_ms * 1e-3) / 1e9
                 # the library's rule (plan_decode): the few-token kernel up to 13 tokens, fewer when few SMs own a neuron tile
                 owners = float(np.mean([(a + 127) // 128 for a in active])) / self.torch.cuda.get_device_properties(0).multi_processor_count
@@ -600,10 +600,10 @@ class Bench:
         return out
 
     def is_one_launch(self, w):
-        """Whether a stack call of workload w is one persistent launch (decode always; prefill when the layers stay in L2)."""
+        """Whether a stack call of workload w is one persistent launch (up to 128 tokens always; prefill when the layers stay in L2)."""
         if not w["stack"]:
             return False
-        return w["n"] <= 64 or 3 * w["d"] * w["I"] * 2 <= (48 << 20)
+        return w["n"] <= 128 or 3 * w["d"] * w["I"] * 2 <= (48 << 20)
 
 
 def run_ours(args):

@@ -222,7 +222,7 @@ mlpmoe_status_t mlpmoe_rmsnorm(const float* x, void* r, int64_t n_tokens, int64_
 /*
  * Set-up of mlpmoe_stack_forward for this stack (these handles, in this order) and this token
  * count, so that the forward call itself only enqueues: chooses the kernel family, builds the work
- * sequences on the host, allocates the device memory that holds them (and, for up to 64 tokens, a
+ * sequences on the host, allocates the device memory that holds them (and, for up to 128 tokens, a
  * stage-tiled copy of each layer's packed weights, as large as the packed weights; if that memory
  * cannot be had, a slower kernel without the copy), uploads them on `stream` and may synchronise
  * `stream`.  The result is cached in the first layer's handle, one set-up at a time: preparing
@@ -238,7 +238,7 @@ mlpmoe_status_t mlpmoe_stack_prepare(const mlpmoe_handle_t* layers, int32_t n_la
  * library-owned buffer of the layer dtype, then x = x + MLPMoE_l(that).
  *
  * bf16 stacks whose layers share one workspace (mlpmoe_share_workspace) run in one
- * persistent kernel: up to 64 tokens always, above 128 tokens when every layer's
+ * persistent kernel: up to 128 tokens always, above 128 tokens when every layer's
  * packed weights are small enough to stay in L2; other stacks run layer by layer.
  * After mlpmoe_stack_prepare for the same stack and token count the call only
  * enqueues: no allocation, no synchronisation.  Without it (or after a create / fade /
@@ -328,7 +328,7 @@ mlpmoe_status_t mlpmoe_get_timing(mlpmoe_handle_t h, double* ms, int64_t* launch
 mlpmoe_status_t mlpmoe_debug_set_wait(mlpmoe_handle_t h, uint64_t limit_ns, uint32_t extra_arrivals);
 
 /*
- * Which persistent kernel a decode stack call (at most 64 tokens) that starts with this layer runs:
+ * Which persistent kernel a decode stack call (at most 128 tokens) that starts with this layer runs:
  * 0 = by the library's rule (token count and how many SMs own a neuron tile), 1 = the few-token kernel
  * (both GEMMs on the tile's owner; at most 16 tokens, more tokens fall back to the rule's other kernel),
  * 2 = the kernel with a grid-wide H exchange.  Both compute the same stack; the tests use this to run

@@ -555,7 +555,7 @@ std::vector<int64_t> stack_key(const mlpmoe_handle_t* layers, int32_t n_layers, 
 // the token operand's tensor map.
 mlpmoe_status_t plan_decode(const mlpmoe_handle_t* layers, int32_t n_layers, int64_t n, cudaStream_t st) {
   mlpmoe_layer_s* h0 = layers[0];
-  const int npad = n <= 16 ? 16 : (n <= 32 ? 32 : 64);
+  const int npad = n <= 16 ? 16 : (n <= 32 ? 32 : (n <= 64 ? 64 : 128));
   bool tiled = true;
   for (int l = 0; tiled && l < n_layers; ++l) {
     mlpmoe_layer_s* h = layers[l];
@@ -659,7 +659,7 @@ mlpmoe_status_t plan_stack(const mlpmoe_handle_t* layers, int32_t n_layers, int6
   h0->plan_kind = PLAN_NONE;
   h0->plan_key.clear();
   int kind = PLAN_PER_LAYER;
-  if (h0->dtype == MLPMOE_BF16 && n <= kDecodeMaxTokens && n_layers <= kMaxStackLayers && h0->d <= 32768 && stack_kernel_ok()) {
+  if (h0->dtype == MLPMOE_BF16 && n <= kDecodeStackMaxTokens && n_layers <= kMaxStackLayers && h0->d <= 32768 && stack_kernel_ok()) {
     // decode: the whole stack in one persistent kernel (weights keep streaming across layer boundaries)
     kind = PLAN_DECODE;
   } else if (h0->dtype == MLPMOE_BF16 && n > 128 && n_layers <= kMaxStackLayers) {

@@ -1,4 +1,4 @@
-// Decode of a whole pre-norm stack (n_tokens <= 64) in ONE persistent, cooperatively launched
+// Decode of a whole pre-norm stack (n_tokens <= 128) in ONE persistent, cooperatively launched
 // kernel: x <- x + MLPMoE_l(RMSNorm(x)) for l = 0 .. L-1.  One CTA per SM; every CTA walks the same
 // static sequence of phases per layer
 //     N: RMSNorm of the token rows into the bf16 activation buffer
@@ -17,7 +17,9 @@
 // otherwise they come from the packed operands through tensor maps.
 //
 // Warp roles: warp 0 TMA producer, warp 1 TMEM owner + MMA issuer, warps 2..5 epilogue (and the
-// RMSNorm phase).  Weights sit on the 128-row side of the MMA, tokens on N = 16 / 32 / 64.
+// RMSNorm phase).  Weights sit on the 128-row side of the MMA, tokens on N = 16 / 32 / 64 / 128.
+// The kernel is built twice: for at most 64 token rows (two accumulator buffers in 256 TMEM columns)
+// and for 128 (all 512 columns).
 #include <cuda_bf16.h>
 
 #include "internal.h"
@@ -31,11 +33,10 @@ using namespace ptx;
 constexpr int BK = 64;
 constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
-constexpr int MAXN = kDecodeMaxTokens;
 constexpr int MAX_STAGES = 6;
 constexpr int W_BYTES = 256 * BK * 2;                 // 256 weight rows per stage in both phases
 // A stage is the weight tile plus a token tile of npad rows; the ring takes as many stages as fit
-// (6 for npad 16 and 32, 5 for npad 64), the barriers sit in front of it.
+// (6 for npad 16 and 32, 5 for npad 64, 4 for npad 128), the barriers sit in front of it.
 constexpr int BAR_BYTES = 1024;
 constexpr int RING_BYTES = 216 * 1024;
 constexpr int SMEM_BYTES = BAR_BYTES + RING_BYTES + 1024;
@@ -44,7 +45,6 @@ __host__ __device__ constexpr int stage_bytes_for(int npad) { return W_BYTES + n
 __host__ __device__ constexpr int stages_for(int npad) {
   return RING_BYTES / stage_bytes_for(npad) < MAX_STAGES ? RING_BYTES / stage_bytes_for(npad) : MAX_STAGES;
 }
-constexpr uint32_t TMEM_COLS = 4 * MAXN;              // 2 buffers x (G | U)
 constexpr uint32_t ARRIVALS_PER_CTA = 1;              // one arrival per CTA and event, after its four epilogue warps have met
 constexpr int NORM_VEC = 8;                           // float4 per lane the RMSNorm phase keeps in registers
 
@@ -83,6 +83,7 @@ __device__ __forceinline__ bool event_wait(const uint32_t* counter, uint32_t tar
 }
 
 // Issues the loads of one accumulator's first npad columns; the values are valid after tmem_ld_wait().
+template <int MAXN>
 __device__ __forceinline__ void load_acc_async(uint32_t taddr, int npad, uint32_t (&v)[MAXN]) {
 #pragma unroll
   for (int c = 0; c < MAXN; c += 16) {
@@ -175,6 +176,7 @@ struct StepIter {
   }
 };
 
+template <int MAXN>                                   // token rows the accumulators hold: 64 or 128
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
                     const __grid_constant__ CUtensorMap tm_x,   // xnorm [n x d] bf16, box 64 x npad
@@ -189,6 +191,7 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   const ClockProbe probe = clock_probe_begin();
+  constexpr uint32_t TMEM_COLS = 4 * MAXN;              // 2 buffers x (G | U)
   volatile float* norm_part = reinterpret_cast<volatile float*>(tmem_slot + 4);   // one partial sum of squares per epilogue warp
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int cta = blockIdx.x, ctas = gridDim.x;
@@ -427,15 +430,20 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
         const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * 2 * MAXN) + (static_cast<uint32_t>(quad * 32) << 16);
 #pragma unroll
         for (int half = 0; half < 2; ++half) {                 // the two blocks of 128 output columns
-          uint32_t v[MAXN];
-          load_acc_async(taddr + half * MAXN, npad, v);
-          tmem_ld_wait();
-          if (half == 1) release_acc();
           const int64_t m = static_cast<int64_t>(it[i].m_blk) * 256 + half * 128 + quad * 32 + lane;
-          if (m < d) {
 #pragma unroll
-            for (int t = 0; t < MAXN; ++t)
-              if (t < n) atomicAdd(x + static_cast<int64_t>(t) * d + m, __uint_as_float(v[t]));
+          for (int c0 = 0; c0 < MAXN; c0 += 64) {              // 64 token rows at a time
+            if (c0 < npad) {
+              uint32_t v[64];
+              load_acc_async(taddr + half * MAXN + c0, npad - c0, v);
+              tmem_ld_wait();
+              if (half == 1 && c0 + 64 >= npad) release_acc();   // the last columns have been read
+              if (m < d) {
+#pragma unroll
+                for (int t = 0; t < 64; ++t)
+                  if (c0 + t < n) atomicAdd(x + static_cast<int64_t>(c0 + t) * d + m, __uint_as_float(v[t]));
+              }
+            }
           }
         }
       }
@@ -453,9 +461,14 @@ decode_stack_kernel(const DecodeStackLayer* __restrict__ layers, int n_layers,
 }  // namespace
 
 cudaError_t decode_stack_init(int* max_ctas_per_sm) {
-  cudaError_t e = cudaFuncSetAttribute(decode_stack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  cudaError_t e = cudaFuncSetAttribute(decode_stack_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_stack_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(max_ctas_per_sm, decode_stack_kernel, NUM_THREADS, SMEM_BYTES);
+  int a = 0, b = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, decode_stack_kernel<64>, NUM_THREADS, SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, decode_stack_kernel<128>, NUM_THREADS, SMEM_BYTES);
+  *max_ctas_per_sm = a < b ? a : b;
+  return e;
 }
 
 // layers_dev: n_layers records in device memory (64-byte aligned).  event_counter: 3 * n_layers zeros.
@@ -469,8 +482,9 @@ cudaError_t launch_decode_stack(const DecodeStackLayer* layers_dev, int n_layers
   void* args[] = {const_cast<DecodeStackLayer**>(&layers_dev), &n_layers, const_cast<CUtensorMap*>(&tm_x), &x, &xn, &n, &d, &npad,
                   &eps, &event_counter, &status, &wait_ns, &extra};
   // cooperative launch: the grid-wide events need every CTA resident at once
-  return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(decode_stack_kernel), dim3(num_sms), dim3(NUM_THREADS), args,
-                                     SMEM_BYTES, st);
+  const void* kernel = npad <= 64 ? reinterpret_cast<const void*>(decode_stack_kernel<64>)
+                                  : reinterpret_cast<const void*>(decode_stack_kernel<128>);
+  return cudaLaunchCooperativeKernel(kernel, dim3(num_sms), dim3(NUM_THREADS), args, SMEM_BYTES, st);
 }
 
 }  // namespace mlpmoe

@@ -40,6 +40,7 @@ constexpr int kGroup = 128;      // neurons per interleaved gate|up group in the
 // the prefill schedules may then re-read them at will instead of streaming them once per group of token blocks.
 constexpr int64_t kWeightsFitL2Bytes = int64_t(48) << 20;
 constexpr int kDecodeMaxTokens = 64;
+constexpr int kDecodeStackMaxTokens = 128;  // most tokens the persistent decode-stack kernel takes (its 128-row build)
 
 // Limits of the bounded waits of one launch.  Ordinary launches use the defaults; the test hook
 // mlpmoe_debug_set_wait shortens the limit and adds `extra_arrivals` to the target of every wait of

@@ -137,10 +137,10 @@ def test_single_branch_and_narrow_survivors(lib, bf16, n):
         lib.mlpmoe_destroy(h)
 
 
-@pytest.mark.parametrize("n,stack,kernel", [(4, True, 1), (4, True, 2), (40, True, 0), (300, True, 0), (300, False, 0)])
+@pytest.mark.parametrize("n,stack,kernel", [(4, True, 1), (4, True, 2), (40, True, 0), (100, True, 0), (300, True, 0), (300, False, 0)])
 def test_bounded_wait_runs_out_and_the_handle_recovers(lib, n, stack, kernel):
-    """The give-up path of the kernels whose CTAs wait for one another (few-token decode stack, 14..64-token
-    decode stack, prefill stack, single-layer prefill): with the wait limit cut to 3 ms and every
+    """The give-up path of the kernels whose CTAs wait for one another (few-token decode stack, the other decode-stack
+    kernel in its 64-row and 128-row builds, prefill stack, single-layer prefill): with the wait limit cut to 3 ms and every
     cross-CTA target raised by one arrival (a count that is never reached) the call must return, the
     status must read DEVICE_TIMEOUT, and, once that has been reported, the same handles must compute
     the right result again.  Nothing traps or faults: the kernels leave their loops and free their TMEM."""

@@ -179,6 +179,37 @@ def destroy(lib, handles):
         lib.mlpmoe_destroy(h)
 
 
+@pytest.mark.parametrize("n", [65, 128])
+def test_llama_shape_decode_stack_65_to_128_tokens(lib, llama_stack, n):
+    """The 128-row build of the persistent decode kernel (65 to 128 tokens) at the Llama shape: three layers, every
+    token row real, against the oracle end to end (3 layers: first-order bound) and on the bulk of the error."""
+    host_bits, dev = llama_stack
+    B, nl = 64, 3
+    d_b = synth.equal_partition(I, B)
+    x = synth.tokens(4, 128, D, stream=7)[:n]
+    handles = []
+    try:
+        for l in range(nl):
+            h = lib.mlpmoe_create(D, I, d_b, dev[l][0], dev[l][1], dev[l][2], None, lib.MLPMOE_BF16, lib.MLPMOE_LAYOUT_PAPER, 128,
+                                  stream_ptr())
+            if handles:
+                lib.mlpmoe_share_workspace(h, handles[0])
+            handles.append(h)
+        layers = [tuple(synth.bf16_bits_to_f32(b) for b in host_bits[l]) + (d_b, [1.0] * B) for l in range(nl)]
+        ref, inputs = oracle.stack_forward(x, layers, bf16_activations=True, return_layer_inputs=True)
+        xd = dev_f32(x)
+        lib.mlpmoe_stack_forward(handles, xd, n, 1e-6, stream_ptr())
+        torch.cuda.synchronize()
+        assert all(lib.mlpmoe_get_status(h) == lib.MLPMOE_OK for h in handles)
+        got = xd.cpu().numpy()
+        tol = stack_tolerance(inputs, ref)
+        e_max, e_rms = rel_err(got, ref), rms_err(got, ref)
+        print(f"{n} tokens, 3 Llama-shaped layers: max|delta|/RMS = {e_max:.4f} (bound {tol:.4f}), RMS(delta)/RMS = {e_rms:.5f}")
+        assert e_max <= tol and e_rms <= 5e-3
+    finally:
+        destroy(lib, handles)
+
+
 def test_config4_decode_stack(lib, llama_stack):
     host_bits, dev = llama_stack
     B = 64
