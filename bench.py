@@ -110,8 +110,8 @@ TRAFFIC = {
     # decode: captured on 4 of the 32 layers; a launch streams its layers' weights once, so traffic scales with the layers
     "llama_decode_1": ((1470823936 + 4195840) * 8, ('decode_fused.cu', 'ptx.cuh'), "41ae9186018dac22", "profiles/decode_fused_kernel_llama_c4_4layers.md"),
     "llama_decode_8": ((1467553280 + 4698368) * 8, ('decode_fused.cu', 'ptx.cuh'), "41ae9186018dac22", "profiles/decode_fused_kernel_llama_c4_4layers.md"),
-    "llama_decode_32": ((1413513472 + 10400768) * 8, ('decode_stack.cu', 'ptx.cuh'), "925b810b9d6e3a09", "profiles/decode_stack_kernel_llama_c4_4layers.md"),
-    "llama_decode_64": ((1416810752 + 15351040) * 8, ('decode_stack.cu', 'ptx.cuh'), "925b810b9d6e3a09", "profiles/decode_stack_kernel_llama_c4_4layers.md"),
+    "llama_decode_32": ((1413492992 + 10519040) * 8, ('decode_stack.cu', 'ptx.cuh'), "73796a8498fd42e1", "profiles/decode_stack_kernel_llama_c4_4layers.md"),
+    "llama_decode_64": ((1416848384 + 15218944) * 8, ('decode_stack.cu', 'ptx.cuh'), "73796a8498fd42e1", "profiles/decode_stack_kernel_llama_c4_4layers.md"),
 }
 
 
